@@ -1,0 +1,117 @@
+/*
+ * ha_la.h -- C ABI of the B200 (sm_100a) delta-rule linear-attention prefill library.
+ *
+ * One operation: the chunkwise-parallel prefill of a Gated DeltaNet (GDN) layer
+ * (scalar log-gate per head per token) or its Kimi-Delta-Attention (KDA)
+ * variant (log-gate per key channel).
+ *
+ * Paper passages that define the operation:
+ *   - Section 2.1, "Architecture of Linear-Attention Hybrids": a fixed-size
+ *     recurrent state per head; at step t the previous state is updated with
+ *     K_t, V_t and the output is formed from Q_t and the UPDATED state.
+ *   - Section 2.1, "Chunkwise Map-Reduce-Map Execution": operators #1 Gate,
+ *     #2 KKT, #3 Solve, #4 W/U (Map), #5 H (Reduce, sequential per head),
+ *     #6 O (Map).  Chunk length 64 (Section "Experimental setup").
+ *   - Section "HA-NPU overview": inputs are Q/K/V, gates and the initial state;
+ *     outputs are the attention outputs and the updated state.
+ *   - Precisions (Section "Experimental setup"): 16-bit Q/K/V, FP32 gates and states.
+ *
+ * Result, per sequence and V-head j (QK-head jq = j / (HV/HK)), with the state
+ * h of shape d_k x d_v starting at h0 (or zero), for each token t in order:
+ *     GDN:  h <- exp(g[t,j]) h            KDA:  h[c,:] <- exp(g[t,j,c]) h[c,:]
+ *     h <- h + beta[t,j] k[t,jq] (v[t,j] - h^T k[t,jq])^T
+ *     o[t,j] = scale * h^T q[t,jq]
+ * and hT = h after the last token.  The library evaluates this chunk by chunk
+ * (chunk = 64); the result does not depend on the chunking beyond rounding.
+ *
+ * Conventions
+ *   - Every pointer in ha_la_prefill_args is a DEVICE pointer owned by the
+ *     caller, valid until the work enqueued on the stream has finished.
+ *   - ha_la_prefill enqueues kernels on the given CUDA stream and returns
+ *     without synchronising.  It allocates no device memory and keeps no
+ *     pointer after it returns; the args struct is read during the call only.
+ *   - Every entry point returns an ha_la_status; nothing throws or aborts.
+ *   - Problems found on the device (a wait that ran out, an index out of
+ *     range) are written as a non-zero code to *status_word, which the caller
+ *     reads after its own synchronisation; the kernels then finish normally
+ *     with unspecified outputs.
+ *   - o must not overlap any input.  hT may be exactly the pointer h0
+ *     (in-place state update) and must not partially overlap it.
+ *   - Sequence lengths need not be multiples of 64; length-0 sequences are
+ *     legal (hT = h0).  Log-gates are expected to be <= 0.
+ */
+#ifndef HA_LA_H_
+#define HA_LA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { HA_LA_GDN = 0, HA_LA_KDA = 1 } ha_la_variant;
+typedef enum { HA_LA_BF16 = 0, HA_LA_FP32 = 1 } ha_la_dtype;   /* dtype of q, k, v and o */
+
+typedef enum {
+  HA_LA_OK = 0,
+  HA_LA_ERR_INVALID_ARG = 1,   /* null pointer, bad size, bad enum                         */
+  HA_LA_ERR_UNSUPPORTED = 2,   /* legal but not implemented (head dim, chunk, ...)         */
+  HA_LA_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small               */
+  HA_LA_ERR_CUDA = 4,          /* a CUDA runtime / driver call or a launch failed          */
+  HA_LA_ERR_TIMEOUT = 5,       /* device side: a bounded wait ran out (status word only)   */
+  HA_LA_ERR_DEVICE_CHECK = 6   /* device side: an index or length check failed             */
+} ha_la_status;
+
+typedef struct {
+  int32_t variant;        /* ha_la_variant                                                   */
+  int32_t dtype;          /* ha_la_dtype                                                     */
+  int32_t batch;          /* B; must be 1 when cu_seqlens != NULL                            */
+  int32_t seqlen;         /* T per batch row; TOTAL packed tokens when cu_seqlens != NULL    */
+  int32_t num_qk_heads;   /* HK                                                              */
+  int32_t num_v_heads;    /* HV, a multiple of HK; V-head j reads QK-head j / (HV/HK)        */
+  int32_t d_k, d_v;       /* 64 or 128 each                                                  */
+  int32_t chunk;          /* must be 64                                                      */
+  float   scale;          /* o = scale * h^T q                                               */
+  const void*  q;         /* [B, T, HK, d_k] contiguous, token-major                         */
+  const void*  k;         /* [B, T, HK, d_k]                                                 */
+  const void*  v;         /* [B, T, HV, d_v]                                                 */
+  const float* g;         /* GDN [B, T, HV]; KDA [B, T, HV, d_k]; log-gate                   */
+  const float* beta;      /* [B, T, HV]                                                      */
+  const float* h0;        /* [N, HV, d_k, d_v] fp32 or NULL (zeros); N = B or num_seqs       */
+  const int32_t* cu_seqlens; /* device int32 [num_seqs+1], cu[0]=0, non-decreasing,
+                                cu[num_seqs]=seqlen; or NULL for B equal-length rows        */
+  int32_t num_seqs;       /* used only when cu_seqlens != NULL                               */
+  int32_t max_seqlen;     /* upper bound on any sequence length when cu_seqlens != NULL
+                             (sizes the launch; a longer sequence is reported through
+                             status_word as HA_LA_ERR_DEVICE_CHECK); 0 = use seqlen          */
+  void*   o;              /* [B, T, HV, d_v], dtype as v                                     */
+  float*  hT;             /* [N, HV, d_k, d_v] fp32 or NULL (not wanted)                     */
+  void*   workspace;      /* >= ha_la_prefill_workspace_bytes(), 256-byte aligned            */
+  size_t  workspace_bytes;
+  int32_t* status_word;   /* optional device int32; the caller zeroes it before the call     */
+} ha_la_prefill_args;
+
+/* Host only: bytes of scratch ha_la_prefill needs for these shapes (pointers are ignored).
+ * Returns HA_LA_OK and writes *out_bytes, or an error for invalid / unsupported shapes.     */
+int ha_la_prefill_workspace_bytes(const ha_la_prefill_args* args, size_t* out_bytes);
+
+/* Enqueue the prefill on `cuda_stream` (a cudaStream_t; NULL = the default stream).
+ * Implements operators #1-#6 of "Chunkwise Map-Reduce-Map Execution" (Section 2.1) for
+ * every sequence and V-head.  Asynchronous; see the conventions above.                     */
+int ha_la_prefill(const ha_la_prefill_args* args, void* cuda_stream);
+
+/* Name of the implementation ha_la_prefill would run for these shapes ("tc" = tcgen05
+ * tensor-core kernels, "simt" = fp32 CUDA-core kernel), or NULL if unsupported.  Host only. */
+const char* ha_la_prefill_path(const ha_la_prefill_args* args);
+
+/* Number of kernels ha_la_prefill launches for these shapes (0 if unsupported).  Host only. */
+int ha_la_prefill_num_launches(const ha_la_prefill_args* args);
+
+const char* ha_la_status_string(int status);
+int ha_la_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HA_LA_H_ */
