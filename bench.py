@@ -1,0 +1,356 @@
+#!/usr/bin/env python
+"""Benchmark of the delta-rule linear-attention prefill library on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" = one pass of the whole hot path (plan + every compute kernel of ha_la_prefill)
+over one batch of the synthetic workload.  Prints ONE JSON line (rank 0).
+
+* value        : tokens/s, inputs resident in HBM, device-timed (CUDA events, max over ranks).
+                 Each step uses a different one of R resident input/output sets whose total
+                 size exceeds 2x the L2 cache, so no step finds its inputs in L2.
+* e2e          : the same metric through the public API with HOST buffers: pinned host -> device
+                 copies of every input and device -> host copies of o and hT inside the timed region.
+* roofline     : for the dominant kernel, timed live with CUDA events between kernels
+                 (ha_la_prefill_timed); `path` gives the spec whole-path figure
+                 (slower of FLOPs at the measured bf16 peak and bytes at the measured HBM rate).
+* cpu_baseline : the fp64 oracle, as it stands, on this machine's host cores, on a bounded sample.
+* --impl reference : times only the oracle (rank 0) and prints its line with "impl": "reference".
+
+With N > 1 (torchrun) every rank runs its own independent batch (the path shards over
+sequences and heads with no exchange): weak scaling, no collective on the data path.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_32114_b200 import synth  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+METRIC = "LA-layer prefill tokens/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_time(inp, budget_heads=None):
+    """Times the oracle on (a sample of) the workload.  Returns (seconds, tokens processed per V-head set,
+    threads, description)."""
+    import oracle
+
+    w = inp["workload"]
+    N = inp["N"]
+    pairs = None
+    desc = f"all {N} sequences x {w.hv} V-heads, every token"
+    if budget_heads is not None and budget_heads < N * w.hv:
+        allp = [(n, j) for n in range(N) for j in range(w.hv)]
+        step = max(1, len(allp) // budget_heads)
+        pairs = allp[::step][:budget_heads]
+        desc = f"{len(pairs)} of {N * w.hv} (sequence, V-head) pairs, every token of each"
+    t0 = time.perf_counter()
+    _, _, threads = oracle.recurrent(inp["q"], inp["k"], inp["v"], inp["g"], inp["beta"], variant=w.variant,
+                                     h0=inp["h0"], cu_seqlens=inp["cu_seqlens"], pairs=pairs)
+    dt = time.perf_counter() - t0
+    if pairs is None:
+        tok_heads = inp["T"] * w.hv
+    else:
+        cu = inp["cu_seqlens"]
+        tok_heads = sum(int(cu[n + 1] - cu[n]) for n, _ in pairs)
+    # tokens/s of the LAYER: token-heads per second divided by heads per token
+    return dt, tok_heads / w.hv, threads, desc
+
+
+def cpu_baseline(inp):
+    w = inp["workload"]
+    # aim at 10-30 s: the recurrence costs about 6 dk dv flops per token-head in fp64
+    work = inp["T"] * w.hv * 6.0 * w.dk * w.dv
+    cores = os.cpu_count() or 1
+    est = work / (cores * 1.0e9)
+    heads = None
+    if est > 25:
+        heads = max(cores, int(inp["N"] * w.hv * 20 / est))
+    dt, tokens, threads, desc = oracle_time(inp, heads)
+    return {"value": tokens / dt, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+            "sample": f"{desc}; {dt:.2f} s wall"}
+
+
+def run_reference(args, inp, rank):
+    """The reference arm of this tier is the oracle itself, timed on the host cores."""
+    if rank != 0:
+        return
+    w = inp["workload"]
+    times = []
+    tokens = threads = None
+    desc = ""
+    work = inp["T"] * w.hv * 6.0 * w.dk * w.dv
+    cores = os.cpu_count() or 1
+    est = work / (cores * 1.0e9)
+    budget = 60.0 / max(1, args.steps + args.warmup)          # keep the whole run within a few minutes
+    heads = None if est <= budget else max(cores, int(inp["N"] * w.hv * budget / est))
+    for i in range(args.warmup + args.steps):
+        dt, tokens, threads, desc = oracle_time(inp, heads)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    val = tokens / (ms / 1e3)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "tokens_per_step": tokens, "sample": desc},
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="gdn_layer_4k", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, synth.make_inputs(w), rank)
+        return
+
+    import torch
+    import paper_2609_32114_b200 as ha
+    from tests import helpers
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    # every rank draws its own batch of the same workload (weak scaling over independent batches)
+    inp = synth.make_inputs(w, seed=synth.BASE_SEED + 1000 * rank)
+    T, N = inp["T"], inp["N"]
+    alg_bytes = synth.algorithmic_bytes(w, T, N)
+    alg_flops = synth.algorithmic_flops(w, T)
+    peaks = load_peaks()
+
+    # R resident buffer sets, total > 2 x L2, visited round-robin
+    base = helpers.to_device(inp, dev)
+    R = max(2, int(np.ceil(2.2 * L2_BYTES / alg_bytes)) + 1)
+    R = min(R, 8)
+    sets = []
+    for r in range(R):
+        d = base if r == 0 else {k: (v.clone() if hasattr(v, "clone") else v) for k, v in base.items()}
+        a, keep = ha.prepare_args(d["q"], d["k"], d["v"], d["g"], d["beta"], variant=w.variant, h0=d["h0"],
+                                  cu_seqlens=d["cu_seqlens"], max_seqlen=d["max_seqlen"])
+        sets.append((a, keep))
+    flush = None
+    if R * alg_bytes < 2 * L2_BYTES:
+        flush = torch.empty(3 * L2_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    sptr = stream.cuda_stream
+    launches_per_step = ha.ha_la_prefill_num_launches(sets[0][0])
+    path = ha.ha_la_prefill_path(sets[0][0])
+
+    def step(i):
+        rc = ha.ha_la_prefill_raw(sets[i % R][0], sptr)
+        if rc != 0:
+            raise ha.HaLaError(rc, "ha_la_prefill")
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    for a, keep in sets:
+        assert int(keep["status_word"].item()) == 0, "device status word set during warm-up"
+
+    # ---- timed region: exactly K steps, device-timed per step (flush, if any, sits outside the events)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    t_wall = time.perf_counter()
+    for i in range(args.steps):
+        if flush is not None:
+            flush.fill_(i & 0xff)
+        evs[i][0].record(stream)
+        step(i)
+        evs[i][1].record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    step_ms = [a.elapsed_time(b) for a, b in evs]
+    total_ms = float(np.sum(step_ms))
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * T / (ms_per_step / 1e3)
+
+    # ---- per-kernel device time (events between kernels), averaged over a few cold-L2 steps
+    kt = {}
+    reps = min(args.steps, 8)
+    for i in range(reps):
+        if flush is not None:
+            flush.fill_(i)
+        for name, ms in ha.ha_la_prefill_timed(sets[(i + 1) % R][0], sptr):
+            kt.setdefault(name, []).append(ms)
+    clocks = sampler.stop()
+    kernel_ms = {k: float(np.mean(v)) for k, v in kt.items()}
+    dom = max(kernel_ms, key=kernel_ms.get)
+    # algorithmic bytes each kernel is the one to touch ("Roofline accounting")
+    e = 2 if w.dtype == "bf16" else 4
+    in_bytes = T * (2 * w.hk * w.dk * e + w.hv * w.dv * e + w.hv * 4 * (1 + (w.dk if w.variant == "kda" else 1)))
+    out_bytes = alg_bytes - in_bytes
+    kernel_alg_bytes = {"simt_prefill": alg_bytes, "tc_prep": in_bytes, "tc_chain": out_bytes, "plan": 0.0}
+    dom_bytes = kernel_alg_bytes.get(dom, alg_bytes)
+    dom_s = kernel_ms[dom] / 1e3
+    achieved = dom_bytes / dom_s / 1e9
+    t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_flop = alg_flops / (peaks["bf16_tflops"] * 1e12)
+    path_s = ms_per_step / 1e3
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "kernel_ms": kernel_ms,
+                "path": {"bound": "hbm" if t_hbm >= t_flop else "tensor", "roofline_us": 1e6 * max(t_hbm, t_flop),
+                         "measured_us": 1e6 * path_s, "frac": max(t_hbm, t_flop) / path_s,
+                         "achieved_gbs": alg_bytes / path_s / 1e9, "achieved_tflops": alg_flops / path_s / 1e12,
+                         "alg_bytes": alg_bytes, "alg_flops": alg_flops}}
+
+    # ---- end to end: pinned host buffers in, o and hT back out, through the public API
+    host = {k: (v.cpu().pin_memory() if hasattr(v, "cpu") else v) for k, v in base.items()}
+    a0, keep0 = sets[0]
+    o_host = torch.empty_like(keep0["o"], device="cpu").pin_memory()
+    hT_host = torch.empty_like(keep0["hT"], device="cpu").pin_memory()
+    names = [k for k in ("q", "k", "v", "g", "beta", "h0", "cu_seqlens") if hasattr(base.get(k), "copy_")]
+    h2d = sum(host[k].numel() * host[k].element_size() for k in names)
+    d2h = o_host.numel() * o_host.element_size() + hT_host.numel() * hT_host.element_size()
+
+    def e2e_step():
+        for k in names:
+            keep0[k].copy_(host[k].view_as(keep0[k]), non_blocking=True)
+        rc = ha.ha_la_prefill_raw(a0, sptr)
+        if rc != 0:
+            raise ha.HaLaError(rc, "ha_la_prefill")
+        o_host.copy_(keep0["o"], non_blocking=True)
+        hT_host.copy_(keep0["hT"], non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e = {"value": world * T / (e2e_ms / args.steps / 1e3), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": int(d2h)}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(inp)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+                "data": "synthetic",
+                "config": {"workload": w.name, "variant": w.variant, "tokens_per_step_per_gpu": T, "sequences": N,
+                           "seq_lens": inp["seq_lens"] if N <= 16 else None, "qk_heads": w.hk, "v_heads": w.hv,
+                           "d_k": w.dk, "d_v": w.dv, "chunk": 64, "path": path,
+                           "l2": f"{R} resident buffer sets visited round-robin ({R * alg_bytes / 1e6:.0f} MB)"
+                                 + (" + L2 flush write between steps" if flush is not None else ""),
+                           "parallelism": "replicas (independent batch per GPU, no collective)" if world > 1 else "1 GPU"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+                "roofline": roofline, "cpu_baseline": cpu, "wall_s_timed_region": t_wall}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -70,7 +70,7 @@ typedef struct {
   int32_t seqlen;         /* T per batch row; TOTAL packed tokens when cu_seqlens != NULL    */
   int32_t num_qk_heads;   /* HK                                                              */
   int32_t num_v_heads;    /* HV, a multiple of HK; V-head j reads QK-head j / (HV/HK)        */
-  int32_t d_k, d_v;       /* 64 or 128 each                                                  */
+  int32_t d_k, d_v;       /* d_k == d_v, 64 or 128                                           */
   int32_t chunk;          /* must be 64                                                      */
   float   scale;          /* o = scale * h^T q                                               */
   const void*  q;         /* [B, T, HK, d_k] contiguous, token-major                         */
@@ -81,7 +81,8 @@ typedef struct {
   const float* h0;        /* [N, HV, d_k, d_v] fp32 or NULL (zeros); N = B or num_seqs       */
   const int32_t* cu_seqlens; /* device int32 [num_seqs+1], cu[0]=0, non-decreasing,
                                 cu[num_seqs]=seqlen; or NULL for B equal-length rows        */
-  int32_t num_seqs;       /* used only when cu_seqlens != NULL                               */
+  int32_t num_seqs;       /* > 0 selects the packed mode and then cu_seqlens is required;
+                             0 with cu_seqlens == NULL means B equal-length rows            */
   int32_t max_seqlen;     /* upper bound on any sequence length when cu_seqlens != NULL
                              (sizes the launch; a longer sequence is reported through
                              status_word as HA_LA_ERR_DEVICE_CHECK); 0 = use seqlen          */
@@ -107,6 +108,14 @@ const char* ha_la_prefill_path(const ha_la_prefill_args* args);
 
 /* Number of kernels ha_la_prefill launches for these shapes (0 if unsupported).  Host only. */
 int ha_la_prefill_num_launches(const ha_la_prefill_args* args);
+
+/* Profiling aid (the paper's "Metrics" paragraph times kernels with device events): the same work
+ * as ha_la_prefill, with a CUDA event recorded on `cuda_stream` before every kernel and after the
+ * last one.  Unlike ha_la_prefill it BLOCKS until the stream has drained, then writes the device
+ * time of each kernel in launch order to ms_out[0..n) (milliseconds), a static name for each to
+ * names_out (may be NULL) and n to *num_kernels_out (n <= max_kernels <= 8).                       */
+int ha_la_prefill_timed(const ha_la_prefill_args* args, void* cuda_stream, int max_kernels, float* ms_out,
+                        const char** names_out, int* num_kernels_out);
 
 const char* ha_la_status_string(int status);
 int ha_la_version(void);

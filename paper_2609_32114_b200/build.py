@@ -1,0 +1,78 @@
+"""Builds libha_la.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
+
+    python -m paper_2609_32114_b200.build [--force] [--verbose]
+
+Objects are cached under paper_2609_32114_b200/build/ and rebuilt when their source, any
+header, or this script changes; translation units compile in parallel.
+"""
+from __future__ import annotations
+
+import concurrent.futures as cf
+import os
+import subprocess
+import sys
+
+PKG = os.path.dirname(os.path.abspath(__file__))
+ROOT = os.path.dirname(PKG)
+CSRC = os.path.join(PKG, "csrc")
+OBJ = os.path.join(PKG, "build")
+LIB = os.path.join(PKG, "libha_la.so")
+INCLUDE = os.path.join(ROOT, "include")
+
+# (object name, source, extra flags)
+UNITS = [("api", "api.cu", []), ("plan", "plan.cu", []), ("tc", "tc.cu", [])] + [
+    (f"simt{u}", "simt.cu", [f"-DHA_LA_SIMT_UNIT={u}"]) for u in range(5)
+]
+ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
+
+
+def _nvcc() -> str:
+    return os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+
+
+def _headers_mtime() -> float:
+    t = os.path.getmtime(os.path.abspath(__file__))
+    for d in (CSRC, INCLUDE):
+        for f in os.listdir(d):
+            if f.endswith((".cuh", ".h")):
+                t = max(t, os.path.getmtime(os.path.join(d, f)))
+    return t
+
+
+def _compile(unit, verbose: bool):
+    name, src, extra = unit
+    out = os.path.join(OBJ, name + ".o")
+    cmd = [_nvcc(), *ARCH, "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC", "-I", CSRC, "-I", INCLUDE,
+           *extra, "-c", os.path.join(CSRC, src), "-o", out]
+    if verbose:
+        cmd += ["-Xptxas", "-v"]
+    r = subprocess.run(cmd, capture_output=True, text=True)
+    return name, r.returncode, r.stdout + r.stderr
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    os.makedirs(OBJ, exist_ok=True)
+    hdr = _headers_mtime()
+    todo = []
+    for unit in UNITS:
+        out = os.path.join(OBJ, unit[0] + ".o")
+        src_t = os.path.getmtime(os.path.join(CSRC, unit[1]))
+        if force or not os.path.exists(out) or os.path.getmtime(out) < max(src_t, hdr):
+            todo.append(unit)
+    if todo:
+        with cf.ThreadPoolExecutor(max_workers=min(len(todo), os.cpu_count() or 4)) as ex:
+            for name, rc, log in ex.map(lambda u: _compile(u, verbose), todo):
+                if verbose or rc != 0:
+                    sys.stderr.write(f"--- {name}\n{log}\n")
+                if rc != 0:
+                    raise RuntimeError(f"nvcc failed on {name}")
+    objs = [os.path.join(OBJ, u[0] + ".o") for u in UNITS]
+    if todo or not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(o) for o in objs):
+        tmp = LIB + f".tmp{os.getpid()}"
+        subprocess.check_call([_nvcc(), *ARCH, "-shared", "-o", tmp, *objs])
+        os.replace(tmp, LIB)
+    return LIB
+
+
+if __name__ == "__main__":
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))

@@ -1,0 +1,89 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, and validates shapes.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2609_32114_b200 as ha
+from paper_2609_32114_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return ha.load_library()
+
+
+def test_exports_match_header(lib):
+    hdr = open(os.path.join(ROOT, "include", "ha_la.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(ha_la_[a-z_]+)\s*\(", hdr))
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+    assert ha.ha_la_version() >= 1
+    assert ha.status_string(0) == "ok" and "workspace" in ha.status_string(3)
+
+
+def test_struct_layout_matches_c(lib):
+    # 10 x 4-byte scalars, 7 pointers, 2 ints, 3 pointers, size_t, pointer on LP64
+    assert ctypes.sizeof(binding.ha_la_prefill_args) == 40 + 7 * 8 + 8 + 3 * 8 + 8 + 8
+    assert binding.ha_la_prefill_args.q.offset == 40
+    assert binding.ha_la_prefill_args.num_seqs.offset == 96
+    assert binding.ha_la_prefill_args.o.offset == 104
+    assert binding.ha_la_prefill_args.workspace_bytes.offset == 128
+
+
+def _args(**kw):
+    base = dict(variant="gdn", dtype="bf16", batch=1, seqlen=4096, hk=16, hv=16, dk=128, dv=128)
+    base.update(kw)
+    return ha.make_args(**base)
+
+
+def test_workspace_query_and_validation(lib):
+    n = ha.ha_la_prefill_workspace_bytes(_args())
+    assert n > 0 and n % 256 == 0
+    n5 = ha.ha_la_prefill_workspace_bytes(_args(seqlen=100000, num_seqs=8))
+    assert n5 >= n
+    assert ha.ha_la_prefill_path(_args(dtype="fp32", dk=64, dv=64, hk=1, hv=1, seqlen=256)) == "simt"
+    assert ha.ha_la_prefill_num_launches(_args()) >= 2
+
+    def status_of(**kw):
+        out = ctypes.c_size_t(0)
+        return lib.ha_la_prefill_workspace_bytes(ctypes.byref(_args(**kw)), ctypes.byref(out))
+
+    assert status_of(variant=7) == binding.HA_LA_ERR_INVALID_ARG
+    assert status_of(dtype=5) == binding.HA_LA_ERR_INVALID_ARG
+    assert status_of(hv=24) == binding.HA_LA_ERR_INVALID_ARG          # not a multiple of hk
+    assert status_of(batch=0) == binding.HA_LA_ERR_INVALID_ARG
+    assert status_of(seqlen=-1) == binding.HA_LA_ERR_INVALID_ARG
+    assert status_of(batch=2, num_seqs=3) == binding.HA_LA_ERR_INVALID_ARG
+    assert status_of(dk=96) == binding.HA_LA_ERR_UNSUPPORTED
+    assert status_of(chunk=32) == binding.HA_LA_ERR_UNSUPPORTED
+    assert status_of(scale=float("nan")) == binding.HA_LA_ERR_INVALID_ARG
+    assert lib.ha_la_prefill_workspace_bytes(None, None) == binding.HA_LA_ERR_INVALID_ARG
+
+
+def test_prefill_rejects_bad_pointers_without_launching(lib):
+    # every check below fails before any CUDA call is made, so this runs without a GPU
+    a = _args()
+    assert binding.ha_la_prefill_raw(a) == binding.HA_LA_ERR_INVALID_ARG       # null q/k/v/...
+    a = _args(q=4096, k=4096, v=4096, g=4096, beta=4096, o=8192)
+    assert binding.ha_la_prefill_raw(a) == binding.HA_LA_ERR_WORKSPACE         # no workspace
+    a = _args(q=4096, k=4096, v=4096, g=4096, beta=4096, o=8192, workspace=4096 + 16, workspace_bytes=1 << 40)
+    assert binding.ha_la_prefill_raw(a) == binding.HA_LA_ERR_WORKSPACE         # misaligned
+    a = _args(q=4096, k=4096, v=4096, g=4096, beta=4096, o=8192, workspace=4096, workspace_bytes=16)
+    assert binding.ha_la_prefill_raw(a) == binding.HA_LA_ERR_WORKSPACE         # too small
+    a = _args(q=4098, k=4096, v=4096, g=4096, beta=4096, o=8192, workspace=4096, workspace_bytes=1 << 40)
+    assert binding.ha_la_prefill_raw(a) == binding.HA_LA_ERR_INVALID_ARG       # q not 16-byte aligned
+    a = _args(q=4096, k=4096, v=4096, g=4096, beta=4096, o=8192, num_seqs=2, workspace=4096, workspace_bytes=1 << 40)
+    assert binding.ha_la_prefill_raw(a) == binding.HA_LA_ERR_INVALID_ARG       # packed mode without cu_seqlens
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    with pytest.raises(FileNotFoundError):
+        ha.load_library(str(tmp_path / "libha_la.so"))

@@ -1,0 +1,145 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU fp64 oracle, element by element,
+on the same seeded inputs.  Tolerances are the spec ones (helpers.TOL): max|err|/max|ref|
+<= 2e-2 for bf16 inputs, <= 1e-4 for fp32, for o and for hT separately."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+from paper_2609_32114_b200 import synth
+from tests import helpers
+
+pytestmark = pytest.mark.gpu
+
+W = synth.WORKLOADS
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2609_32114_b200 import build
+    build.build()
+
+
+def test_config1_gdn_fp32_exact_shape():
+    inp = synth.make_inputs(W["gdn_fp32_small"])
+    res = helpers.check_parity(inp)
+    assert res["o_err"] < 1e-4 and res["hT_err"] < 1e-4
+
+
+@pytest.mark.parametrize("T", [1, 63, 64, 65, 1000])
+def test_gdn_bf16_small_ragged(T):
+    w = synth.shrink(W["gdn_layer_4k"], seq_lens=[T], hk=2, hv=2)
+    helpers.check_parity(synth.make_inputs(w, seed=11 + T))
+
+
+@pytest.mark.parametrize("gate_shift", [-4.0, None])
+def test_gdn_bf16_slow_decay(gate_shift):
+    """Slow or no decay keeps old chunks visible, which is what exercises the inter-chunk state."""
+    w = synth.shrink(W["gdn_layer_4k"], seq_lens=[1500], hk=2, hv=2, gate_shift=gate_shift or 0.0, h0_std=0.02)
+    inp = synth.make_inputs(w, seed=5)
+    if gate_shift is None:
+        inp["g"][:] = 0
+    helpers.check_parity(inp)
+
+
+def test_gdn_fp32_d128_and_scale():
+    w = dataclasses.replace(W["gdn_fp32_small"], dk=128, dv=128, seq_lens=(300,), hk=2, hv=2, h0_std=0.02)
+    helpers.check_parity(synth.make_inputs(w, seed=3), scale=0.25)
+
+
+def test_gva_small():
+    w = synth.shrink(W["gdn_gva_16k"], seq_lens=[700], hk=2, hv=4)
+    helpers.check_parity(synth.make_inputs(w, seed=7))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_kda_small(dtype):
+    w = synth.shrink(W["kda_8k"], seq_lens=[330], hk=2, hv=2, dtype=dtype, h0_std=0.02)
+    helpers.check_parity(synth.make_inputs(w, seed=9))
+
+
+def test_kda_slow_decay():
+    w = synth.shrink(W["kda_8k"], seq_lens=[700], hk=1, hv=2, gate_shift=-4.0)
+    helpers.check_parity(synth.make_inputs(w, seed=10))
+
+
+def test_varlen_small_with_empty_and_tiny_sequences():
+    w = synth.shrink(W["gdn_varlen"], seq_lens=[70, 0, 129, 64, 5, 1, 600], hk=2, hv=2)
+    inp = synth.make_inputs(w, seed=13)
+    o, hT, status = helpers.run_gpu(inp)
+    assert status == 0
+    np.testing.assert_array_equal(hT[1], inp["h0"][1].astype(np.float64))     # empty sequence: hT = h0
+    helpers.check_parity(inp)
+
+
+def test_batched_equal_length_rows():
+    w = synth.shrink(W["gdn_layer_4k"], seq_lens=[200, 200, 200], hk=2, hv=2, h0_std=0.02)
+    helpers.check_parity(synth.make_inputs(w, seed=17))
+
+
+def test_split_resume_and_in_place_state():
+    """Prefill [0,T1) then [T1,T) with h0 := hT (same buffer) equals one call: only the state crosses."""
+    import torch
+    import paper_2609_32114_b200 as ha
+
+    w = synth.shrink(W["gdn_layer_4k"], seq_lens=[500], hk=2, hv=2)
+    inp = synth.make_inputs(w, seed=19)
+    d = helpers.to_device(inp)
+    o_full, hT_full, st, _ = ha.ha_la_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"])
+    T1 = 203
+    cut = lambda t, a, b: t[:, a:b].contiguous()
+    state = torch.zeros_like(hT_full)
+    oa, _, st1, _ = ha.ha_la_prefill(*(cut(d[x], 0, T1) for x in ("q", "k", "v", "g", "beta")), h0=state, hT=state)
+    ob, _, st2, _ = ha.ha_la_prefill(*(cut(d[x], T1, 500) for x in ("q", "k", "v", "g", "beta")), h0=state, hT=state)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and int(st1.item()) == 0 and int(st2.item()) == 0
+    o_split = torch.cat([oa, ob], dim=1).float().cpu().numpy()
+    o_ref = o_full.float().cpu().numpy()
+    scale_o = np.abs(o_ref).max()
+    assert np.abs(o_split - o_ref).max() / scale_o <= 2e-2
+    h_ref = hT_full.cpu().numpy()
+    assert np.abs(state.cpu().numpy() - h_ref).max() / np.abs(h_ref).max() <= 2e-2
+
+
+def test_run_to_run_determinism():
+    w = synth.shrink(W["gdn_layer_4k"], seq_lens=[777], hk=2, hv=4)
+    inp = synth.make_inputs(w, seed=23)
+    o1, h1, _ = helpers.run_gpu(inp)
+    o2, h2, _ = helpers.run_gpu(inp)
+    np.testing.assert_array_equal(o1, o2)
+    np.testing.assert_array_equal(h1, h2)
+
+
+def test_bad_cu_seqlens_reports_device_check():
+    import torch
+
+    w = synth.shrink(W["gdn_varlen"], seq_lens=[100, 50], hk=1, hv=1)
+    inp = synth.make_inputs(w, seed=29)
+    inp["cu_seqlens"] = np.array([0, 120, 100], dtype=np.int32)     # decreasing; last entry != T
+    o, hT, status = helpers.run_gpu(inp)
+    assert status == 6                                               # HA_LA_ERR_DEVICE_CHECK
+    torch.cuda.synchronize()
+
+
+# ---------------------------------------------------------------- full-size configurations, sampled heads
+
+def _pairs_for(inp, heads):
+    lens = inp["seq_lens"]
+    if len(lens) == 1:
+        return [(0, h) for h in heads]
+    order = np.argsort(lens)
+    return [(int(order[-1]), heads[0]), (int(order[0]), heads[-1]), (int(order[len(order) // 2]), heads[1])]
+
+
+@pytest.mark.parametrize("name,heads", [
+    ("gdn_layer_4k", [0, 7, 15]),
+    ("gdn_gva_16k", [1, 30]),
+    ("kda_8k", [0, 31]),
+    ("gdn_varlen", [0, 5, 15]),
+])
+def test_full_size_sampled(name, heads):
+    """Full-size workload in the launch configuration the bench times; the oracle evaluates a sample
+    of (sequence, V-head) pairs in full (every token of those heads)."""
+    inp = synth.make_inputs(W[name])
+    res = helpers.check_parity(inp, pairs=_pairs_for(inp, heads))
+    print(name, res)
