@@ -60,7 +60,8 @@ typedef enum {
   HA_LA_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small               */
   HA_LA_ERR_CUDA = 4,          /* a CUDA runtime / driver call or a launch failed          */
   HA_LA_ERR_TIMEOUT = 5,       /* device side: a bounded wait ran out (status word only)   */
-  HA_LA_ERR_DEVICE_CHECK = 6   /* device side: an index or length check failed             */
+  HA_LA_ERR_DEVICE_CHECK = 6,  /* device side: an index or length check failed             */
+  HA_LA_ERR_TOO_LARGE = 7      /* ha_la_prefill_noalloc only: problem exceeds its fixed scratch */
 } ha_la_status;
 
 typedef struct {
@@ -116,6 +117,29 @@ int ha_la_prefill_num_launches(const ha_la_prefill_args* args);
  * names_out (may be NULL) and n to *num_kernels_out (n <= max_kernels <= 8).                       */
 int ha_la_prefill_timed(const ha_la_prefill_args* args, void* cuda_stream, int max_kernels, float* ms_out,
                         const char** names_out, int* num_kernels_out);
+
+/* Prefill without a workspace, for callers that cannot allocate device memory or hand scratch to
+ * this library (an operator hook that must stay out of its framework's allocator, a runtime whose
+ * memory pool is frozen, a plug-in that only sees the operator's own tensors).  The paper has no
+ * counterpart of this entry point; it computes exactly what ha_la_prefill computes.
+ *
+ *   - args->workspace and args->workspace_bytes are ignored.  The chunk table lives in a fixed
+ *     array inside the library image (ha_la_prefill_noalloc_scratch_bytes() bytes, about 208 KiB),
+ *     which every GPU that loads the library holds until the process exits.
+ *   - Limits: at most 1024 sequences (batch rows or packed sequences) and at most 16384 chunk
+ *     slots ((seqlen + 63 * num_seqs) / 64 in packed mode, batch * ceil(seqlen / 64) otherwise);
+ *     beyond that it returns HA_LA_ERR_TOO_LARGE and launches nothing.
+ *   - It always runs the fp32 CUDA-core kernels (the tensor-core path needs megabytes of scratch),
+ *     so it is meant for small and medium problems; results agree with ha_la_prefill within the
+ *     library's tolerances.
+ *   - It calls no cudaMalloc / cudaFree and no allocating library routine.  Its FIRST call on a
+ *     device looks up the array's device address (cudaGetSymbolAddress, with that device current)
+ *     and caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to start at zero (each call
+ *     rewrites every entry it later reads), but two calls that overlap on the GPU -- different
+ *     streams without an ordering between them -- race on it: serialise them.                     */
+int ha_la_prefill_noalloc(const ha_la_prefill_args* args, void* cuda_stream);
+size_t ha_la_prefill_noalloc_scratch_bytes(void);
 
 const char* ha_la_status_string(int status);
 int ha_la_version(void);

@@ -11,6 +11,8 @@ from .binding import (  # noqa: F401
     ha_la_prefill_args,
     ha_la_prefill_num_launches,
     ha_la_prefill_path,
+    ha_la_prefill_noalloc,
+    ha_la_prefill_noalloc_scratch_bytes,
     ha_la_prefill_raw,
     ha_la_prefill_timed,
     ha_la_prefill_workspace_bytes,

@@ -18,6 +18,7 @@ HA_LA_ERR_WORKSPACE = 3
 HA_LA_ERR_CUDA = 4
 HA_LA_ERR_TIMEOUT = 5
 HA_LA_ERR_DEVICE_CHECK = 6
+HA_LA_ERR_TOO_LARGE = 7
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libha_la.so")
@@ -26,6 +27,8 @@ EXPORTS = (
     "ha_la_prefill_workspace_bytes",
     "ha_la_prefill",
     "ha_la_prefill_timed",
+    "ha_la_prefill_noalloc",
+    "ha_la_prefill_noalloc_scratch_bytes",
     "ha_la_prefill_path",
     "ha_la_prefill_num_launches",
     "ha_la_status_string",
@@ -90,6 +93,10 @@ def load_library(path: Optional[str] = None):
     lib.ha_la_prefill_timed.argtypes = [A, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_float),
                                         ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_int)]
     lib.ha_la_prefill_timed.restype = ctypes.c_int
+    lib.ha_la_prefill_noalloc.argtypes = [A, ctypes.c_void_p]
+    lib.ha_la_prefill_noalloc.restype = ctypes.c_int
+    lib.ha_la_prefill_noalloc_scratch_bytes.argtypes = []
+    lib.ha_la_prefill_noalloc_scratch_bytes.restype = ctypes.c_size_t
     lib.ha_la_prefill_path.argtypes = [A]
     lib.ha_la_prefill_path.restype = ctypes.c_char_p
     lib.ha_la_prefill_num_launches.argtypes = [A]
@@ -143,6 +150,16 @@ def ha_la_prefill_num_launches(args: ha_la_prefill_args) -> int:
 def ha_la_prefill_raw(args: ha_la_prefill_args, stream: int = 0) -> int:
     """The C call itself; returns the status code."""
     return load_library().ha_la_prefill(ctypes.byref(args), ctypes.c_void_p(stream) if stream else None)
+
+
+def ha_la_prefill_noalloc(args: ha_la_prefill_args, stream: int = 0) -> int:
+    """The C call for callers that cannot supply scratch memory (the workspace fields are ignored);
+    returns the status code.  See include/ha_la.h for its limits and its sharing rules."""
+    return load_library().ha_la_prefill_noalloc(ctypes.byref(args), ctypes.c_void_p(stream) if stream else None)
+
+
+def ha_la_prefill_noalloc_scratch_bytes() -> int:
+    return load_library().ha_la_prefill_noalloc_scratch_bytes()
 
 
 def ha_la_prefill_timed(args: ha_la_prefill_args, stream: int = 0):

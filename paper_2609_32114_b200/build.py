@@ -20,7 +20,8 @@ LIB = os.path.join(PKG, "libha_la.so")
 INCLUDE = os.path.join(ROOT, "include")
 
 # (object name, source, extra flags)
-UNITS = [("api", "api.cu", []), ("plan", "plan.cu", []), ("tc", "tc.cu", [])] + [
+UNITS = [("api", "api.cu", []), ("plan", "plan.cu", []), ("tc", "tc.cu", []),
+         ("noalloc", "noalloc.cu", [])] + [
     (f"simt{u}", "simt.cu", [f"-DHA_LA_SIMT_UNIT={u}"]) for u in range(5)
 ]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]

@@ -160,6 +160,7 @@ const char* ha_la_status_string(int status) {
     case HA_LA_ERR_CUDA: return "CUDA call or kernel launch failed";
     case HA_LA_ERR_TIMEOUT: return "device-side wait ran out";
     case HA_LA_ERR_DEVICE_CHECK: return "device-side check failed";
+    case HA_LA_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of ha_la_prefill_noalloc";
     default: return "unknown status";
   }
 }
