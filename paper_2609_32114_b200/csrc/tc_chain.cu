@@ -1,0 +1,316 @@
+// Sequential part of the delta-rule prefill on tcgen05 tensor cores: operator #5 (state passing)
+// with operator #6 (output) fused in the paper's chunk-first order.
+//
+// One CTA per (sequence, V-head, slice of NV value channels) walks the chunks of its sequence in
+// order.  The d_k x NV slice of the state stays on chip for the whole sequence: fp32 in registers
+// (thread t owns key channel t), plus a bf16 copy in shared memory as the MMA operand.  Value
+// channels are independent (paper Section "Computation Splitting": the state splits column-wise
+// into sub-heads with no cross-core reduction), so slices never communicate.
+//
+// Per chunk, with the operand images the prep kernel left in the workspace:
+//   MMA1  D1[128 x NV] = [W ; Q~] h          rows 0..63: W h, rows 64..127: Q~ h      (M = 128)
+//         threads 0..63  : U~_i = (U_i - (W h)_i) e^{G_L - G_i}  -> bf16 operand in shared memory
+//         threads 64..127: o_i  = scale (O_loc,i + (Q~ h)_i)     -> global memory (op #6, uses the OLD state)
+//   MMA2  D2[128 x NV] = K^T U~              (A = the raw K tile, feature-major, by TMA)
+//         all threads    : h <- e^{G_L} h + D2                   (op #5 update, in place)
+// A producer warp keeps the next chunks' operands in flight (1-D bulk copies + one TMA tile) through
+// a ring of shared-memory stages guarded by full/empty mbarriers; every wait is bounded.
+#include <cuda.h>
+
+#include "tc_common.cuh"
+#include "tc_ptx.cuh"
+
+namespace ha_la {
+
+using namespace ptx;
+
+namespace {
+
+constexpr int kChainThreads = 160;       // 4 compute warps + 1 producer warp
+
+template <int NV> struct ChainCfg {
+  static constexpr int kStages = NV == 128 ? 2 : 3;
+  static constexpr uint32_t kRowB = NV * 2;                      // bytes of one operand row (NV bf16)
+  static constexpr uint32_t kSliceB = NV * 128;                  // bytes of an NV-row slice of an image
+  static constexpr uint32_t OFF_WQ = 0;                          // 32 KiB
+  static constexpr uint32_t OFF_K = 32768;                       // 16 KiB  [kb][64 tok][64 feat]
+  static constexpr uint32_t OFF_U = 49152;                       // NV rows of the U image
+  static constexpr uint32_t OFF_O = OFF_U + kSliceB;             // NV rows of the O_loc image
+  static constexpr uint32_t OFF_SC = OFF_O + kSliceB;            // 192 floats
+  static constexpr uint32_t kStageB = (OFF_SC + 768 + 1023) / 1024 * 1024;
+  static constexpr uint32_t kTxBytes = 32768 + 16384 + 2 * kSliceB + 768;
+  static constexpr uint32_t OFF_H = kStages * kStageB;           // bf16 h operand [128][NV]
+  static constexpr uint32_t OFF_UT = OFF_H + 128 * kRowB;        // bf16 U~ operand [64][NV]
+  static constexpr uint32_t OFF_BAR = OFF_UT + 64 * kRowB;
+  static constexpr uint32_t kSmem = OFF_BAR + 128;
+  static constexpr uint32_t kTmemCols = 2 * NV < 32 ? 32 : 2 * NV;
+};
+
+struct ChainParams {
+  const float* h0;
+  float* hT;
+  void* o;
+  const int32_t* seq_tok0;
+  const int32_t* seq_len;
+  const int32_t* seq_chunk0;
+  TcWorkspace ws;
+  int HK, HV;
+  float scale;
+  int32_t* status;
+};
+
+// MN-major B operand with ROWS rows (K index) of NV bf16 each.  NV = 32: 64-byte rows, 64-byte swizzle.
+// NV = 64: 128-byte rows, 128-byte swizzle.  NV = 128: two such 64-column blocks, ROWS*128 bytes apart.
+template <int NV, int ROWS> __device__ __forceinline__ uint32_t brow_offset(int row, int ch) {
+  if (NV == 32) return sw64_offset(row, ch);
+  return static_cast<uint32_t>(ch >> 3) * (ROWS * 128u) + sw128_offset(row, ch & 7);
+}
+template <int NV, int ROWS> __device__ __forceinline__ uint64_t brow_desc(uint32_t base, int kstep) {
+  if (NV == 32) return smem_desc(base + kstep * 16 * 64, 16, 512, kSwizzle64B);
+  return smem_desc(base + kstep * 2048, ROWS * 128, 1024, kSwizzle128B);
+}
+
+// 32 consecutive columns [c0, c0+32) of one operand row
+template <int NV, int ROWS>
+__device__ __forceinline__ void store_brow32(uint8_t* tile, int row, int c0, const float (&v)[32]) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint4 w;
+    w.x = pack_bf16(v[q * 8 + 0], v[q * 8 + 1]);
+    w.y = pack_bf16(v[q * 8 + 2], v[q * 8 + 3]);
+    w.z = pack_bf16(v[q * 8 + 4], v[q * 8 + 5]);
+    w.w = pack_bf16(v[q * 8 + 6], v[q * 8 + 7]);
+    *reinterpret_cast<uint4*>(tile + brow_offset<NV, ROWS>(row, (c0 >> 3) + q)) = w;
+  }
+}
+
+__device__ __forceinline__ void ld32f(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  tmem_ld32(taddr, r);
+  tmem_ld_wait();
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void compute_sync() {     // the 128 compute threads only
+  asm volatile("bar.sync 1, 128;" ::: "memory");
+}
+
+template <int NV>
+__global__ void __launch_bounds__(kChainThreads, 1)
+tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
+  using Cfg = ChainCfg<NV>;
+  constexpr int S = Cfg::kStages;
+  constexpr int NSL = 128 / NV;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bar_full = reinterpret_cast<uint64_t*>(sm + Cfg::OFF_BAR);     // [S]
+  uint64_t* bar_empty = bar_full + S;                                       // [S]
+  uint64_t* bar_mma = bar_empty + S;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mma + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const int slice = blockIdx.x % NSL;
+  const int nj = blockIdx.x / NSL;
+  const int j = nj % p.HV, n = nj / p.HV;
+  const int jq = j / (p.HV / p.HK);
+  const int tok0 = p.seq_tok0[n];
+  const int len = p.seq_len[n];
+  const int chunk0 = p.seq_chunk0[n];
+  const int nchunks = (len + kChunk - 1) / kChunk;
+
+  if (tid == 0) {
+    for (int i = 0; i < S; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 1); }
+    mbar_init(bar_mma, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tmap(&map_k);
+  }
+  if (warp == 0) tmem_alloc(tmem_slot, Cfg::kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------ producer
+    if ((tid & 31) == 0) {
+      for (int c = 0; c < nchunks; ++c) {
+        const int st = c % S;
+        if (c >= S) mbar_wait(&bar_empty[st], ((c / S) - 1) & 1, abort_flag);
+        uint8_t* stage = sm + st * Cfg::kStageB;
+        const size_t cj = (size_t)(chunk0 + c) * p.HV + j;
+        mbar_expect_tx(&bar_full[st], Cfg::kTxBytes);
+        bulk_load(stage + Cfg::OFF_WQ, p.ws.wq + cj * 2 * kImgBytes, 32768, &bar_full[st]);
+        tma_load_3d(stage + Cfg::OFF_K, &map_k, &bar_full[st], 0, jq, tok0 + c * kChunk);
+        tma_load_3d(stage + Cfg::OFF_K + 8192, &map_k, &bar_full[st], 64, jq, tok0 + c * kChunk);
+        bulk_load(stage + Cfg::OFF_U, p.ws.u + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
+        bulk_load(stage + Cfg::OFF_O, p.ws.ol + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
+        bulk_load(stage + Cfg::OFF_SC, p.ws.sc + cj * kScFloats, 768, &bar_full[st]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ compute (threads 0..127)
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t TM1 = tmem, TM2 = tmem + NV;
+    uint8_t* sH = sm + Cfg::OFF_H;
+    uint8_t* sUt = sm + Cfg::OFF_UT;
+
+    float h[NV];                                         // state row `tid` (key channel), NV value channels
+    {
+      const size_t base = (((size_t)n * p.HV + j) * 128 + tid) * 128 + (size_t)slice * NV;
+#pragma unroll
+      for (int q = 0; q < NV; q += 4) {
+        float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (p.h0) v4 = *reinterpret_cast<const float4*>(p.h0 + base + q);
+        h[q] = v4.x; h[q + 1] = v4.y; h[q + 2] = v4.z; h[q + 3] = v4.w;
+      }
+    }
+#pragma unroll
+    for (int c0 = 0; c0 < NV; c0 += 32) {
+      float t[32];
+#pragma unroll
+      for (int q = 0; q < 32; ++q) t[q] = h[c0 + q];
+      store_brow32<NV, 128>(sH, tid, c0, t);
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    compute_sync();
+
+    uint32_t mma_phase = 0;
+    for (int c = 0; c < nchunks; ++c) {
+      const int st = c % S;
+      const uint8_t* stage = sm + st * Cfg::kStageB;
+      const int L = min(kChunk, len - c * kChunk);
+
+      // ---- MMA1: D1 = [W ; Q~] h
+      if (tid == 0) {
+        mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
+        tc_fence_after_sync();
+        const uint32_t id = idesc_bf16(128, NV, true, true);
+        const uint32_t a = smem_u32(stage + Cfg::OFF_WQ);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          umma_ss(TM1, smem_desc(a + ks * 2048, 16384, 1024, kSwizzle128B), brow_desc<NV, 128>(smem_u32(sH), ks), id, ks > 0);
+        umma_commit(bar_mma);
+      }
+      if (tid != 0) mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);   // every reader of the stage observes it
+      mbar_wait(bar_mma, mma_phase, abort_flag);
+      mma_phase ^= 1;
+      tc_fence_after_sync();
+      {
+        const int i = tid & 63;
+        const uint8_t* img = stage + (tid < 64 ? Cfg::OFF_U : Cfg::OFF_O);
+        const float dec = reinterpret_cast<const float*>(stage + Cfg::OFF_SC)[i];
+        __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
+                              ((size_t)(tok0 + c * kChunk + i) * p.HV + j) * 128 + (size_t)slice * NV;
+#pragma unroll
+        for (int c0 = 0; c0 < NV; c0 += 32) {
+          float d[32];
+          ld32f(TM1 + lane_base + c0, d);
+          if (tid < 64) {                                  // U~ rows: (U - W h) e^{G_L - G_i}
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+              const __nv_bfloat16 u =
+                  *reinterpret_cast<const __nv_bfloat16*>(img + sw128_offset(c0 + q, i >> 3) + (i & 7) * 2);
+              d[q] = (__bfloat162float(u) - d[q]) * dec;
+            }
+            store_brow32<NV, 64>(sUt, i, c0, d);
+          } else {                                         // output rows: scale (O_loc + Q~ h)
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+              const __nv_bfloat16 u =
+                  *reinterpret_cast<const __nv_bfloat16*>(img + sw128_offset(c0 + q, i >> 3) + (i & 7) * 2);
+              d[q] = p.scale * (__bfloat162float(u) + d[q]);
+            }
+            if (i < L) {
+#pragma unroll
+              for (int q = 0; q < 32; q += 8) {
+                uint4 w;
+                w.x = pack_bf16(d[q + 0], d[q + 1]); w.y = pack_bf16(d[q + 2], d[q + 3]);
+                w.z = pack_bf16(d[q + 4], d[q + 5]); w.w = pack_bf16(d[q + 6], d[q + 7]);
+                *reinterpret_cast<uint4*>(orow + c0 + q) = w;
+              }
+            }
+          }
+        }
+      }
+      fence_proxy_async_smem();
+      tc_fence_before_sync();
+      compute_sync();
+
+      // ---- MMA2: D2 = K^T U~
+      if (tid == 0) {
+        tc_fence_after_sync();
+        const uint32_t id = idesc_bf16(128, NV, true, true);
+        const uint32_t a = smem_u32(stage + Cfg::OFF_K);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          umma_ss(TM2, smem_desc(a + ks * 2048, 8192, 1024, kSwizzle128B), brow_desc<NV, 64>(smem_u32(sUt), ks), id, ks > 0);
+        umma_commit(bar_mma);
+      }
+      const float gam = reinterpret_cast<const float*>(stage + Cfg::OFF_SC)[64 + tid];
+      mbar_wait(bar_mma, mma_phase, abort_flag);
+      mma_phase ^= 1;
+      tc_fence_after_sync();
+#pragma unroll
+      for (int c0 = 0; c0 < NV; c0 += 32) {
+        float d[32];
+        ld32f(TM2 + lane_base + c0, d);
+#pragma unroll
+        for (int q = 0; q < 32; ++q) {
+          h[c0 + q] = fmaf(gam, h[c0 + q], d[q]);
+          d[q] = h[c0 + q];
+        }
+        store_brow32<NV, 128>(sH, tid, c0, d);
+      }
+      fence_proxy_async_smem();
+      tc_fence_before_sync();
+      compute_sync();
+      if (tid == 0) mbar_arrive(&bar_empty[st]);         // every compute thread is done with this stage
+    }
+
+    if (p.hT) {
+      const size_t base = (((size_t)n * p.HV + j) * 128 + tid) * 128 + (size_t)slice * NV;
+#pragma unroll
+      for (int q = 0; q < NV; q += 4)
+        *reinterpret_cast<float4*>(p.hT + base + q) = make_float4(h[q], h[q + 1], h[q + 2], h[q + 3]);
+    }
+  }
+
+  if (*abort_flag && tid == 0) report_status(p.status, HA_LA_ERR_TIMEOUT);
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
+}
+
+template <int NV>
+cudaError_t launch_nv(const ChainParams& cp, const CUtensorMap& mk, int grid, cudaStream_t stream) {
+  auto kern = tc_chain_kernel<NV>;
+  const int smem = ChainCfg<NV>::kSmem + 1024;
+  static_assert(ChainCfg<NV>::kSmem + 1024 <= 227 * 1024, "shared memory budget");
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  timer_mark(stream, "tc_chain");
+  kern<<<grid, kChainThreads, smem, stream>>>(mk, cp);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
+                            const CUtensorMap& mk, int nv, cudaStream_t stream) {
+  ChainParams cp;
+  cp.h0 = a.h0; cp.hT = a.hT; cp.o = a.o;
+  cp.seq_tok0 = plan.seq_tok0; cp.seq_len = plan.seq_len; cp.seq_chunk0 = plan.seq_chunk0;
+  cp.ws = ws; cp.HK = p.HK; cp.HV = p.HV; cp.scale = p.scale; cp.status = a.status_word;
+  const int grid = p.N * p.HV * (128 / nv);
+  if (grid == 0) return cudaSuccess;
+  if (nv == 32) return launch_nv<32>(cp, mk, grid, stream);
+  if (nv == 64) return launch_nv<64>(cp, mk, grid, stream);
+  return launch_nv<128>(cp, mk, grid, stream);
+}
+
+}  // namespace ha_la

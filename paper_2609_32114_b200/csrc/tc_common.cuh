@@ -1,0 +1,42 @@
+// Layout of the tensor-core path's workspace and the parameters shared by its two kernels.
+//
+// For every (chunk slot s, V-head j), cj = s * HV + j, the prep kernel writes
+//   wq  [cj] : 32 KiB  W image (16 KiB) followed by the Q~ image (16 KiB)
+//   u   [cj] : 16 KiB  U image
+//   ol  [cj] : 16 KiB  O_loc image
+//   sc  [cj] : 192 floats  e^{G_L - G_i} for the 64 tokens, then e^{G_L} for the 128 key channels
+// An "image" is a 128 x 64 bf16 matrix stored feature-major: row r (key or value channel) holds the
+// 64 tokens of the chunk in 128 bytes, and the eight 16-byte pieces of a row are stored at piece
+// index (p XOR (r mod 8)).  That is byte for byte the 128-byte-swizzled shared-memory layout that
+// tcgen05.mma reads, so the chain kernel fetches images with plain 1-D bulk copies.
+#pragma once
+
+#include "common.cuh"
+
+namespace ha_la {
+
+constexpr size_t kImgBytes = 128 * 64 * 2;     // 16 KiB
+constexpr int kScFloats = 192;
+
+struct TcWorkspace {
+  uint8_t* wq;
+  uint8_t* u;
+  uint8_t* ol;
+  float* sc;
+};
+
+inline __host__ size_t tc_ws_bytes_for(size_t ncj) {
+  return ncj * (2 * kImgBytes + kImgBytes + kImgBytes) + align_up(ncj * kScFloats * sizeof(float), 1024);
+}
+
+inline __host__ TcWorkspace tc_ws_view(void* base, size_t ncj) {
+  TcWorkspace w;
+  uint8_t* b = reinterpret_cast<uint8_t*>(base);
+  w.wq = b;                      b += ncj * 2 * kImgBytes;
+  w.u = b;                       b += ncj * kImgBytes;
+  w.ol = b;                      b += ncj * kImgBytes;
+  w.sc = reinterpret_cast<float*>(b);
+  return w;
+}
+
+}  // namespace ha_la

@@ -143,3 +143,16 @@ def test_full_size_sampled(name, heads):
     inp = synth.make_inputs(W[name])
     res = helpers.check_parity(inp, pairs=_pairs_for(inp, heads))
     print(name, res)
+
+
+@pytest.mark.parametrize("nv", [32, 64, 128])
+def test_tc_every_slice_width(nv, monkeypatch):
+    """The tensor-core chain kernel at each value-slice width (normally chosen from the launch size)."""
+    import paper_2609_32114_b200 as ha
+
+    monkeypatch.setenv("HA_LA_TC_NV", str(nv))
+    w = synth.shrink(W["gdn_varlen"], seq_lens=[130, 700, 64], hk=2, hv=4, gate_shift=-1.0)
+    inp = synth.make_inputs(w, seed=31 + nv)
+    a = ha.make_args(variant="gdn", dtype="bf16", batch=1, seqlen=inp["T"], hk=2, hv=4, dk=128, dv=128, num_seqs=3)
+    assert ha.ha_la_prefill_path(a) == "tc"
+    helpers.check_parity(inp)
