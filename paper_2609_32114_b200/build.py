@@ -40,9 +40,10 @@ def _headers_mtime() -> float:
     return t
 
 
-def _compile(unit, verbose: bool):
+def _compile(unit, verbose: bool, obj_dir: str = OBJ, more=()):
     name, src, extra = unit
-    out = os.path.join(OBJ, name + ".o")
+    extra = list(extra) + list(more)
+    out = os.path.join(obj_dir, name + ".o")
     cmd = [_nvcc(), *ARCH, "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC", "-I", CSRC, "-I", INCLUDE,
            *extra, "-c", os.path.join(CSRC, src), "-o", out]
     if verbose:
@@ -51,28 +52,29 @@ def _compile(unit, verbose: bool):
     return name, r.returncode, r.stdout + r.stderr
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, extra_flags=(), lib_path: str = LIB, obj_dir: str = OBJ) -> str:
+    """Compile what is stale and link.  `extra_flags`, `lib_path`, `obj_dir` serve developer builds."""
+    os.makedirs(obj_dir, exist_ok=True)
     hdr = _headers_mtime()
     todo = []
     for unit in UNITS:
-        out = os.path.join(OBJ, unit[0] + ".o")
+        out = os.path.join(obj_dir, unit[0] + ".o")
         src_t = os.path.getmtime(os.path.join(CSRC, unit[1]))
         if force or not os.path.exists(out) or os.path.getmtime(out) < max(src_t, hdr):
             todo.append(unit)
     if todo:
         with cf.ThreadPoolExecutor(max_workers=min(len(todo), os.cpu_count() or 4)) as ex:
-            for name, rc, log in ex.map(lambda u: _compile(u, verbose), todo):
+            for name, rc, log in ex.map(lambda u: _compile(u, verbose, obj_dir, extra_flags), todo):
                 if verbose or rc != 0:
                     sys.stderr.write(f"--- {name}\n{log}\n")
                 if rc != 0:
                     raise RuntimeError(f"nvcc failed on {name}")
-    objs = [os.path.join(OBJ, u[0] + ".o") for u in UNITS]
-    if todo or not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(o) for o in objs):
-        tmp = LIB + f".tmp{os.getpid()}"
+    objs = [os.path.join(obj_dir, u[0] + ".o") for u in UNITS]
+    if todo or not os.path.exists(lib_path) or os.path.getmtime(lib_path) < max(os.path.getmtime(o) for o in objs):
+        tmp = lib_path + f".tmp{os.getpid()}"
         subprocess.check_call([_nvcc(), *ARCH, "-shared", "-o", tmp, *objs])
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib_path)
+    return lib_path
 
 
 if __name__ == "__main__":

@@ -8,6 +8,7 @@ using namespace ha_la;
 
 namespace ha_la { thread_local KernelTimer* g_timer = nullptr; }
 
+
 namespace {
 
 bool dim_ok(int d) { return d == 64 || d == 128; }
@@ -83,10 +84,16 @@ const char* ha_la_prefill_path(const ha_la_prefill_args* args) {
   return use_tc(p) ? "tc" : "simt";
 }
 
+// The chunk table is only needed for packed batches and by the CUDA-core kernel; the tensor-core
+// kernels index equal-length rows arithmetically.
+static bool needs_plan(const ha_la_prefill_args* a, const Problem& p) {
+  return a->num_seqs > 0 || a->cu_seqlens != nullptr || !use_tc(p);
+}
+
 int ha_la_prefill_num_launches(const ha_la_prefill_args* args) {
   Problem p;
   if (make_problem(args, &p) != HA_LA_OK) return 0;
-  return 1 + (use_tc(p) ? tc_num_launches(p) : 1);
+  return (needs_plan(args, p) ? 1 : 0) + (use_tc(p) ? tc_num_launches(p) : 1);
 }
 
 int ha_la_prefill(const ha_la_prefill_args* a, void* cuda_stream) {
@@ -109,7 +116,11 @@ int ha_la_prefill(const ha_la_prefill_args* a, void* cuda_stream) {
 
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   PlanView plan = plan_view(a->workspace, p);
-  if (launch_plan(p, a->cu_seqlens, plan, a->status_word, stream) != cudaSuccess) return HA_LA_ERR_CUDA;
+  if (needs_plan(a, p)) {
+    if (launch_plan(p, a->cu_seqlens, plan, a->status_word, stream) != cudaSuccess) return HA_LA_ERR_CUDA;
+  } else {
+    plan = PlanView{};                                   // null table: equal-length rows, indexed arithmetically
+  }
   if (p.T_total == 0 && !a->hT) return HA_LA_OK;
 
   cudaError_t e;

@@ -1,0 +1,17 @@
+// Optional phase timestamps for kernel tuning.  Compiled in only with -DHA_LA_PROFILE_PHASES (a
+// developer build); in the normal build both macros expand to nothing.
+#pragma once
+#ifdef HA_LA_PROFILE_PHASES
+#define HA_PROF_DECL(name)                                                                        \
+  static __device__ long long g_prof_##name[1024];                                                \
+  extern "C" int ha_la_debug_read_prof_##name(long long* out) {                                   \
+    return cudaMemcpyFromSymbol(out, g_prof_##name, sizeof(long long) * 1024) == cudaSuccess ? 0 : 4; \
+  }
+#define HA_PROF(name, slot)                                                            \
+  do {                                                                                 \
+    if (threadIdx.x == 0 && blockIdx.x == 0 && (slot) < 1024) g_prof_##name[slot] = clock64(); \
+  } while (0)
+#else
+#define HA_PROF_DECL(name)
+#define HA_PROF(name, slot) do { } while (0)
+#endif

@@ -7,7 +7,8 @@
 namespace ha_la {
 
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream);
+                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int nv,
+                           cudaStream_t stream);
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                             const CUtensorMap& mk, int nv, cudaStream_t stream);
 
@@ -81,9 +82,10 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
       !make_map(&mv, a.v, p.T_total, p.HV))
     return cudaErrorInvalidValue;
   const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV);
-  cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, stream);
+  const int nv = pick_nv(p);
+  cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, nv, stream);
   if (e != cudaSuccess) return e;
-  return launch_tc_chain(p, a, plan, ws, mk, pick_nv(p), stream);
+  return launch_tc_chain(p, a, plan, ws, mk, nv, stream);
 }
 
 }  // namespace ha_la

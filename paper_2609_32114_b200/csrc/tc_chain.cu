@@ -13,29 +13,37 @@
 //         threads 64..127: o_i  = scale (O_loc,i + (Q~ h)_i)     -> global memory (op #6, uses the OLD state)
 //   MMA2  D2[128 x NV] = K^T U~              (A = the raw K tile, feature-major, by TMA)
 //         all threads    : h <- e^{G_L} h + D2                   (op #5 update, in place)
-// A producer warp keeps the next chunks' operands in flight (1-D bulk copies + one TMA tile) through
-// a ring of shared-memory stages guarded by full/empty mbarriers; every wait is bounded.
+//
+// Warp roles: warps 0-3 compute (thread t <-> tensor-memory lane t), warp 4 produces (keeps the next
+// chunks' operands in flight through a ring of shared-memory stages: 1-D bulk copies + one TMA
+// tile), warp 5 issues the MMAs.  A tcgen05.mma costs the issuing thread about 65 cycles whatever
+// its N <= 128, so issue runs on its own warp and is told "operand ready" with arrive-only named
+// barriers; the compute warps never wait for issue, only for completion (mbarriers).  Every
+// mbarrier wait is bounded.
 #include <cuda.h>
 
 #include "tc_common.cuh"
 #include "tc_ptx.cuh"
+#include "prof.cuh"
 
 namespace ha_la {
 
 using namespace ptx;
 
+HA_PROF_DECL(chain)
+
 namespace {
 
-constexpr int kChainThreads = 160;       // 4 compute warps + 1 producer warp
+constexpr int kChainThreads = 192;       // 4 compute warps + producer warp + MMA warp
 
 template <int NV> struct ChainCfg {
   static constexpr int kStages = NV == 128 ? 2 : 3;
   static constexpr uint32_t kRowB = NV * 2;                      // bytes of one operand row (NV bf16)
-  static constexpr uint32_t kSliceB = NV * 128;                  // bytes of an NV-row slice of an image
+  static constexpr uint32_t kSliceB = NV * 128;                  // bytes of one 64 x NV export tile
   static constexpr uint32_t OFF_WQ = 0;                          // 32 KiB
   static constexpr uint32_t OFF_K = 32768;                       // 16 KiB  [kb][64 tok][64 feat]
-  static constexpr uint32_t OFF_U = 49152;                       // NV rows of the U image
-  static constexpr uint32_t OFF_O = OFF_U + kSliceB;             // NV rows of the O_loc image
+  static constexpr uint32_t OFF_U = 49152;                       // 64 x NV tile of U
+  static constexpr uint32_t OFF_O = OFF_U + kSliceB;             // 64 x NV tile of O_loc
   static constexpr uint32_t OFF_SC = OFF_O + kSliceB;            // 192 floats
   static constexpr uint32_t kStageB = (OFF_SC + 768 + 1023) / 1024 * 1024;
   static constexpr uint32_t kTxBytes = 32768 + 16384 + 2 * kSliceB + 768;
@@ -50,9 +58,10 @@ struct ChainParams {
   const float* h0;
   float* hT;
   void* o;
-  const int32_t* seq_tok0;
-  const int32_t* seq_len;
+  const int32_t* seq_tok0;     // per-sequence table of the plan kernel, or NULL for equal-length rows
+  const int32_t* seq_len;      //   (then sequence n is tokens [n*T_row, (n+1)*T_row), cps chunk slots each)
   const int32_t* seq_chunk0;
+  int T_row, cps;
   TcWorkspace ws;
   int HK, HV;
   float scale;
@@ -65,10 +74,12 @@ template <int NV, int ROWS> __device__ __forceinline__ uint32_t brow_offset(int 
   if (NV == 32) return sw64_offset(row, ch);
   return static_cast<uint32_t>(ch >> 3) * (ROWS * 128u) + sw128_offset(row, ch & 7);
 }
-template <int NV, int ROWS> __device__ __forceinline__ uint64_t brow_desc(uint32_t base, int kstep) {
-  if (NV == 32) return smem_desc(base + kstep * 16 * 64, 16, 512, kSwizzle64B);
-  return smem_desc(base + kstep * 2048, ROWS * 128, 1024, kSwizzle128B);
+// Descriptor of k-step 0; k-step ks (16 rows further) adds ks * brow_step16<NV>() to the start-address field.
+template <int NV, int ROWS> __device__ __forceinline__ uint64_t brow_desc0(uint32_t base) {
+  if (NV == 32) return smem_desc(base, 16, 512, kSwizzle64B);
+  return smem_desc(base, ROWS * 128, 1024, kSwizzle128B);
 }
+template <int NV> __host__ __device__ constexpr uint32_t brow_step16() { return (NV == 32 ? 16u * 64u : 2048u) >> 4; }
 
 // 32 consecutive columns [c0, c0+32) of one operand row
 template <int NV, int ROWS>
@@ -83,6 +94,19 @@ __device__ __forceinline__ void store_brow32(uint8_t* tile, int row, int c0, con
     *reinterpret_cast<uint4*>(tile + brow_offset<NV, ROWS>(row, (c0 >> 3) + q)) = w;
   }
 }
+template <int NV, int ROWS>
+__device__ __forceinline__ void load_brow32(const uint8_t* tile, int row, int c0, float (&v)[32]) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint4 w = *reinterpret_cast<const uint4*>(tile + brow_offset<NV, ROWS>(row, (c0 >> 3) + q));
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      v[q * 8 + 2 * e] = __uint_as_float(u[e] << 16);
+      v[q * 8 + 2 * e + 1] = __uint_as_float(u[e] & 0xffff0000u);
+    }
+  }
+}
 
 __device__ __forceinline__ void ld32f(uint32_t taddr, float (&v)[32]) {
   uint32_t r[32];
@@ -92,8 +116,14 @@ __device__ __forceinline__ void ld32f(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-__device__ __forceinline__ void compute_sync() {     // the 128 compute threads only
-  asm volatile("bar.sync 1, 128;" ::: "memory");
+// named barriers (0 is __syncthreads)
+constexpr int BAR_H_READY = 1;   // 128 compute threads arrive, MMA warp syncs: bf16 h is in shared memory
+constexpr int BAR_U_READY = 2;   // 64 U~ writers arrive, MMA warp syncs: U~ operand is in shared memory
+__device__ __forceinline__ void named_arrive(int id, int count) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void named_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
 template <int NV>
@@ -104,10 +134,11 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   constexpr int NSL = 128 / NV;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bar_full = reinterpret_cast<uint64_t*>(sm + Cfg::OFF_BAR);     // [S]
-  uint64_t* bar_empty = bar_full + S;                                       // [S]
-  uint64_t* bar_mma = bar_empty + S;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mma + 1);
+  uint64_t* bar_full = reinterpret_cast<uint64_t*>(sm + Cfg::OFF_BAR);     // [S]  producer -> everyone
+  uint64_t* bar_empty = bar_full + S;                                       // [S]  128 compute threads -> producer
+  uint64_t* bar_mma1 = bar_empty + S;                                       // MMA1 complete
+  uint64_t* bar_mma2 = bar_mma1 + 1;                                        // MMA2 complete
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mma2 + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x;
@@ -116,14 +147,15 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   const int nj = blockIdx.x / NSL;
   const int j = nj % p.HV, n = nj / p.HV;
   const int jq = j / (p.HV / p.HK);
-  const int tok0 = p.seq_tok0[n];
-  const int len = p.seq_len[n];
-  const int chunk0 = p.seq_chunk0[n];
+  const int tok0 = p.seq_tok0 ? p.seq_tok0[n] : n * p.T_row;
+  const int len = p.seq_tok0 ? p.seq_len[n] : p.T_row;
+  const int chunk0 = p.seq_tok0 ? p.seq_chunk0[n] : n * p.cps;
   const int nchunks = (len + kChunk - 1) / kChunk;
 
   if (tid == 0) {
-    for (int i = 0; i < S; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 1); }
-    mbar_init(bar_mma, 1);
+    for (int i = 0; i < S; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 128); }
+    mbar_init(bar_mma1, 1);
+    mbar_init(bar_mma2, 1);
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&map_k);
@@ -133,6 +165,9 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
+  const uint32_t TM1 = tmem, TM2 = tmem + NV;
+  uint8_t* sH = sm + Cfg::OFF_H;
+  uint8_t* sUt = sm + Cfg::OFF_UT;
 
   if (warp == 4) {
     // ------------------------------------------------------------ producer
@@ -144,20 +179,45 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
         const size_t cj = (size_t)(chunk0 + c) * p.HV + j;
         mbar_expect_tx(&bar_full[st], Cfg::kTxBytes);
         bulk_load(stage + Cfg::OFF_WQ, p.ws.wq + cj * 2 * kImgBytes, 32768, &bar_full[st]);
-        tma_load_3d(stage + Cfg::OFF_K, &map_k, &bar_full[st], 0, jq, tok0 + c * kChunk);
-        tma_load_3d(stage + Cfg::OFF_K + 8192, &map_k, &bar_full[st], 64, jq, tok0 + c * kChunk);
         bulk_load(stage + Cfg::OFF_U, p.ws.u + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
         bulk_load(stage + Cfg::OFF_O, p.ws.ol + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
         bulk_load(stage + Cfg::OFF_SC, p.ws.sc + cj * kScFloats, 768, &bar_full[st]);
+        tma_load_3d(stage + Cfg::OFF_K, &map_k, &bar_full[st], 0, jq, tok0 + c * kChunk);
+        tma_load_3d(stage + Cfg::OFF_K + 8192, &map_k, &bar_full[st], 64, jq, tok0 + c * kChunk);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------ MMA issue (lane 0 issues; the warp keeps the barriers)
+    const uint32_t id = idesc_bf16(128, NV, true, true);
+    const uint64_t dH = brow_desc0<NV, 128>(smem_u32(sH));
+    const uint64_t dU = brow_desc0<NV, 64>(smem_u32(sUt));
+    const bool lead = (tid & 31) == 0;
+    for (int c = 0; c < nchunks; ++c) {
+      const int st = c % S;
+      const uint32_t stage = smem_u32(sm + st * Cfg::kStageB);
+      const uint64_t dWQ = smem_desc(stage + Cfg::OFF_WQ, 16384, 1024, kSwizzle128B);
+      const uint64_t dK = smem_desc(stage + Cfg::OFF_K, 8192, 1024, kSwizzle128B);
+      if (lead) mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
+      named_sync(BAR_H_READY, 128 + 32);                 // h (bf16) of the previous chunk is in sH
+      if (lead) {
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)                    // K = d_k: 16 feature rows (2048 B) per step
+          umma_ss(TM1, dWQ + ks * (2048u >> 4), dH + ks * brow_step16<NV>(), id, ks > 0);
+        umma_commit(bar_mma1);
+      }
+      named_sync(BAR_U_READY, 64 + 32);                  // U~ is in sUt
+      if (lead) {
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)                    // K = tokens: 16 token rows per step
+          umma_ss(TM2, dK + ks * (2048u >> 4), dU + ks * brow_step16<NV>(), id, ks > 0);
+        umma_commit(bar_mma2);
       }
     }
   } else {
     // ------------------------------------------------------------ compute (threads 0..127)
     const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
-    const uint32_t TM1 = tmem, TM2 = tmem + NV;
-    uint8_t* sH = sm + Cfg::OFF_H;
-    uint8_t* sUt = sm + Cfg::OFF_UT;
-
     float h[NV];                                         // state row `tid` (key channel), NV value channels
     {
       const size_t base = (((size_t)n * p.HV + j) * 128 + tid) * 128 + (size_t)slice * NV;
@@ -177,84 +237,68 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
-    compute_sync();
+    named_arrive(BAR_H_READY, 128 + 32);
 
-    uint32_t mma_phase = 0;
+    const int i = tid & 63;                              // token row handled in the first epilogue
     for (int c = 0; c < nchunks; ++c) {
       const int st = c % S;
       const uint8_t* stage = sm + st * Cfg::kStageB;
       const int L = min(kChunk, len - c * kChunk);
+      const uint32_t ph = c & 1;
 
-      // ---- MMA1: D1 = [W ; Q~] h
-      if (tid == 0) {
-        mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
-        tc_fence_after_sync();
-        const uint32_t id = idesc_bf16(128, NV, true, true);
-        const uint32_t a = smem_u32(stage + Cfg::OFF_WQ);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_ss(TM1, smem_desc(a + ks * 2048, 16384, 1024, kSwizzle128B), brow_desc<NV, 128>(smem_u32(sH), ks), id, ks > 0);
-        umma_commit(bar_mma);
-      }
-      if (tid != 0) mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);   // every reader of the stage observes it
-      mbar_wait(bar_mma, mma_phase, abort_flag);
-      mma_phase ^= 1;
+      HA_PROF(chain, 8 * c + 0);
+      mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
+      HA_PROF(chain, 8 * c + 1);
+      // operands of the first epilogue that do not depend on the MMA, fetched while it runs
+      const float* sc = reinterpret_cast<const float*>(stage + Cfg::OFF_SC);
+      const float dec = sc[i];
+      const float gam = sc[64 + tid];
+      float pre[32];
+      load_brow32<NV, 64>(stage + (tid < 64 ? Cfg::OFF_U : Cfg::OFF_O), i, 0, pre);
+
+      mbar_wait(bar_mma1, ph, abort_flag);
+      HA_PROF(chain, 8 * c + 2);
       tc_fence_after_sync();
-      {
-        const int i = tid & 63;
-        const uint8_t* img = stage + (tid < 64 ? Cfg::OFF_U : Cfg::OFF_O);
-        const float dec = reinterpret_cast<const float*>(stage + Cfg::OFF_SC)[i];
+      if (tid < 64) {                                    // U~ rows: (U - W h) e^{G_L - G_i}, the MMA2 operand
+#pragma unroll
+        for (int c0 = 0; c0 < NV; c0 += 32) {
+          float d[32];
+          ld32f(TM1 + lane_base + c0, d);
+          if (c0 > 0) load_brow32<NV, 64>(stage + Cfg::OFF_U, i, c0, pre);
+#pragma unroll
+          for (int q = 0; q < 32; ++q) d[q] = (pre[q] - d[q]) * dec;
+          store_brow32<NV, 64>(sUt, i, c0, d);
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        named_arrive(BAR_U_READY, 64 + 32);
+        HA_PROF(chain, 8 * c + 3);
+      } else {                                           // output rows: o = scale (O_loc + Q~ h)  (op #6)
         __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
                               ((size_t)(tok0 + c * kChunk + i) * p.HV + j) * 128 + (size_t)slice * NV;
 #pragma unroll
         for (int c0 = 0; c0 < NV; c0 += 32) {
           float d[32];
           ld32f(TM1 + lane_base + c0, d);
-          if (tid < 64) {                                  // U~ rows: (U - W h) e^{G_L - G_i}
+          if (c0 > 0) load_brow32<NV, 64>(stage + Cfg::OFF_O, i, c0, pre);
 #pragma unroll
-            for (int q = 0; q < 32; ++q) {
-              const __nv_bfloat16 u =
-                  *reinterpret_cast<const __nv_bfloat16*>(img + sw128_offset(c0 + q, i >> 3) + (i & 7) * 2);
-              d[q] = (__bfloat162float(u) - d[q]) * dec;
-            }
-            store_brow32<NV, 64>(sUt, i, c0, d);
-          } else {                                         // output rows: scale (O_loc + Q~ h)
+          for (int q = 0; q < 32; ++q) d[q] = p.scale * (pre[q] + d[q]);
+          if (i < L) {
 #pragma unroll
-            for (int q = 0; q < 32; ++q) {
-              const __nv_bfloat16 u =
-                  *reinterpret_cast<const __nv_bfloat16*>(img + sw128_offset(c0 + q, i >> 3) + (i & 7) * 2);
-              d[q] = p.scale * (__bfloat162float(u) + d[q]);
-            }
-            if (i < L) {
-#pragma unroll
-              for (int q = 0; q < 32; q += 8) {
-                uint4 w;
-                w.x = pack_bf16(d[q + 0], d[q + 1]); w.y = pack_bf16(d[q + 2], d[q + 3]);
-                w.z = pack_bf16(d[q + 4], d[q + 5]); w.w = pack_bf16(d[q + 6], d[q + 7]);
-                *reinterpret_cast<uint4*>(orow + c0 + q) = w;
-              }
+            for (int q = 0; q < 32; q += 8) {
+              uint4 w;
+              w.x = pack_bf16(d[q + 0], d[q + 1]); w.y = pack_bf16(d[q + 2], d[q + 3]);
+              w.z = pack_bf16(d[q + 4], d[q + 5]); w.w = pack_bf16(d[q + 6], d[q + 7]);
+              *reinterpret_cast<uint4*>(orow + c0 + q) = w;
             }
           }
         }
       }
-      fence_proxy_async_smem();
-      tc_fence_before_sync();
-      compute_sync();
 
-      // ---- MMA2: D2 = K^T U~
-      if (tid == 0) {
-        tc_fence_after_sync();
-        const uint32_t id = idesc_bf16(128, NV, true, true);
-        const uint32_t a = smem_u32(stage + Cfg::OFF_K);
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          umma_ss(TM2, smem_desc(a + ks * 2048, 8192, 1024, kSwizzle128B), brow_desc<NV, 64>(smem_u32(sUt), ks), id, ks > 0);
-        umma_commit(bar_mma);
-      }
-      const float gam = reinterpret_cast<const float*>(stage + Cfg::OFF_SC)[64 + tid];
-      mbar_wait(bar_mma, mma_phase, abort_flag);
-      mma_phase ^= 1;
+      mbar_wait(bar_mma2, ph, abort_flag);
+      HA_PROF(chain, 8 * c + 4);
       tc_fence_after_sync();
+      mbar_arrive(&bar_empty[st]);                       // this thread and both MMAs are done with the stage
 #pragma unroll
       for (int c0 = 0; c0 < NV; c0 += 32) {
         float d[32];
@@ -268,8 +312,8 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
       }
       fence_proxy_async_smem();
       tc_fence_before_sync();
-      compute_sync();
-      if (tid == 0) mbar_arrive(&bar_empty[st]);         // every compute thread is done with this stage
+      named_arrive(BAR_H_READY, 128 + 32);
+      HA_PROF(chain, 8 * c + 5);
     }
 
     if (p.hT) {
@@ -280,6 +324,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
     }
   }
 
+  if (warp == 5) named_sync(BAR_H_READY, 128 + 32);      // pairs with the compute warps' last arrival
   if (*abort_flag && tid == 0) report_status(p.status, HA_LA_ERR_TIMEOUT);
   tc_fence_before_sync();
   __syncthreads();
@@ -305,6 +350,7 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   ChainParams cp;
   cp.h0 = a.h0; cp.hT = a.hT; cp.o = a.o;
   cp.seq_tok0 = plan.seq_tok0; cp.seq_len = plan.seq_len; cp.seq_chunk0 = plan.seq_chunk0;
+  cp.T_row = p.T_row; cp.cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
   cp.ws = ws; cp.HK = p.HK; cp.HV = p.HV; cp.scale = p.scale; cp.status = a.status_word;
   const int grid = p.N * p.HV * (128 / nv);
   if (grid == 0) return cudaSuccess;

@@ -1,17 +1,19 @@
 // Chunk-local operators of the delta-rule prefill on tcgen05 tensor cores (GDN).
 //
-// One CTA per (chunk slot, V-head).  Implements, for its chunk (paper Section 2.1, "Chunkwise
-// Map-Reduce-Map Execution"):
+// One CTA (8 warps) per (chunk slot, V-head).  Implements, for its chunk (paper Section 2.1,
+// "Chunkwise Map-Reduce-Map Execution"):
 //   #1 Gate   G = chunk-local cumulative log-gate (warp scan)
 //   #2 KKT    S = [K; Q] K^T on the tensor cores (one M=128 MMA covers K K^T and Q K^T), then
 //             A_ij = beta_i e^{G_i-G_j} S_kk[i,j] (j<i)  and  P_ij = e^{G_i-G_j} S_qk[i,j] (j<=i) in fp32
-//   #3 Solve  T = (I + A)^-1 in fp32: two 32x32 diagonal blocks by forward substitution, the
-//             off-diagonal block as -T_11 (A_10 T_00)
+//   #3 Solve  T = (I + A)^-1 in fp32 by blocked forward substitution: four 16x16 diagonal blocks,
+//             then the off-diagonal blocks level by level as T_lo = -T_hi (A_lo T_lo')
 //   #4 W/U    W^T = K^T (T diag(beta e^G))^T,  U^T = V^T (T diag(beta))^T   (M = feature dim = 128)
 // and the chunk-local halves of operator #6, so that the sequential kernel needs one stacked MMA:
 //             Q~ = Q e^G - P W      O_loc = P U        (o = scale [Q~ h + O_loc])
-// Operands arrive by TMA (bf16, 128-byte swizzle), accumulators live in tensor memory, results go
-// to the workspace as ready-to-use operand images (tc_common.cuh).
+// Operands arrive by TMA (bf16, 128-byte swizzle), accumulators live in tensor memory, results are
+// assembled in shared memory as ready-to-use operand images (tc_common.cuh) and leave by bulk copy.
+//
+// Warp w reads tensor-memory lanes 32*(w%4)..+31 (accumulator rows) and columns 32*(w/4)..+31.
 //
 // Tokens past the end of a sequence are made no-ops by beta = 0 and g = 0; whatever the TMA box
 // read for them (the next sequence's rows, or zero fill past the end of the tensor) is multiplied
@@ -20,21 +22,24 @@
 
 #include "tc_common.cuh"
 #include "tc_ptx.cuh"
+#include "prof.cuh"
 
 namespace ha_la {
 
 using namespace ptx;
 
+HA_PROF_DECL(prep)
+
 namespace {
 
-constexpr int kPrepThreads = 128;
+constexpr int kPrepThreads = 256;
 constexpr int LDF = 68;                  // row stride (floats) of the fp32 64x64 matrices
 constexpr int LDX = 36;                  // row stride of the 32x32 scratch
 
 // shared-memory map (bytes from the 1024-aligned base)
 constexpr uint32_t OFF_KQ = 0;           // [kb][K 8K | Q 8K], kb = 0,1 (feature halves)
-constexpr uint32_t OFF_V = 32768;        // [kb][V 8K]
-constexpr uint32_t OFF_R1 = 49152;       // solve scratch, later the W^T / U^T operand tiles
+constexpr uint32_t OFF_V = 32768;        // [kb][V 8K]; later the Q~ image
+constexpr uint32_t OFF_R1 = 49152;       // solve scratch, later the W^T / U^T operand tiles (= W, U images)
 constexpr uint32_t OFF_A = OFF_R1;                       // fp32 [64][LDF]; later T^W, T^U tiles
 constexpr uint32_t OFF_T = OFF_R1 + 64 * LDF * 4;        // fp32 [64][LDF]
 constexpr uint32_t OFF_X = OFF_T + 64 * LDF * 4;         // fp32 [32][LDX]
@@ -52,34 +57,50 @@ static_assert(OFF_UT + 16384 <= OFF_P, "operand tiles overlap P");
 struct PrepParams {
   const float* g;
   const float* beta;
-  const int32_t* chunk_tok0;
-  const int32_t* chunk_len;
+  const int32_t* chunk_tok0;   // chunk table of the plan kernel, or NULL for equal-length rows:
+  const int32_t* chunk_len;    //   then slot s is chunk s % cps of row s / cps, T_row tokens per row
+  int T_row, cps;
   TcWorkspace ws;
   int HK, HV;
+  int nv;                 // value channels per chain CTA (32, 64 or 128): layout of the U / O_loc exports
   int32_t* status;
 };
 
-__device__ __forceinline__ void ld64(uint32_t taddr, float (&v)[64]) {
-  uint32_t r0[32], r1[32];
-  tmem_ld32(taddr, r0);
-  tmem_ld32(taddr + 32, r1);
+__device__ __forceinline__ void ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  tmem_ld32(taddr, r);
   tmem_ld_wait();
 #pragma unroll
-  for (int i = 0; i < 32; ++i) { v[i] = __uint_as_float(r0[i]); v[32 + i] = __uint_as_float(r1[i]); }
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// 64 fp32 values of one feature row -> eight 16-byte pieces of bf16, swizzled, to shared and/or global
-__device__ __forceinline__ void store_row_image(const float (&v)[64], int row, uint8_t* smem_tile, uint8_t* gmem_img) {
+// 32 fp32 values (columns 32*hf .. +31 of one 64-column row) -> four 16-byte pieces of bf16, swizzled
+__device__ __forceinline__ void store_half_row(const float (&v)[32], int row, int hf, uint8_t* tile) {
 #pragma unroll
-  for (int ch = 0; ch < 8; ++ch) {
+  for (int q = 0; q < 4; ++q) {
     uint4 w;
-    w.x = pack_bf16(v[ch * 8 + 0], v[ch * 8 + 1]);
-    w.y = pack_bf16(v[ch * 8 + 2], v[ch * 8 + 3]);
-    w.z = pack_bf16(v[ch * 8 + 4], v[ch * 8 + 5]);
-    w.w = pack_bf16(v[ch * 8 + 6], v[ch * 8 + 7]);
-    const uint32_t off = sw128_offset(row, ch);
-    if (smem_tile) *reinterpret_cast<uint4*>(smem_tile + off) = w;
-    if (gmem_img) *reinterpret_cast<uint4*>(gmem_img + off) = w;
+    w.x = pack_bf16(v[q * 8 + 0], v[q * 8 + 1]);
+    w.y = pack_bf16(v[q * 8 + 2], v[q * 8 + 3]);
+    w.z = pack_bf16(v[q * 8 + 4], v[q * 8 + 5]);
+    w.w = pack_bf16(v[q * 8 + 6], v[q * 8 + 7]);
+    *reinterpret_cast<uint4*>(tile + sw128_offset(row, hf * 4 + q)) = w;
+  }
+}
+
+// Scatter 32 token values of feature row `r` (tokens 32*hf .. +31) into a token-major export: for each slice
+// of `nv` value channels a 64 x nv bf16 tile in the chain kernel's row layout (64-byte rows with the 64-byte
+// swizzle for nv = 32, else 128-byte rows with the 128-byte swizzle, 64 channels per 8 KiB block).
+// `region(b)` maps export byte b to shared memory.
+template <typename Region>
+__device__ __forceinline__ void store_token_major(const float (&v)[32], int r, int hf, int nv, Region region) {
+  const int slice = r / nv, col = r % nv;
+  const uint32_t base = static_cast<uint32_t>(slice) * nv * 128 + (col & 7) * 2;
+  const int ch = col >> 3;
+#pragma unroll
+  for (int q = 0; q < 32; ++q) {
+    const int i = hf * 32 + q;
+    const uint32_t off = nv == 32 ? sw64_offset(i, ch) : static_cast<uint32_t>(ch >> 3) * 8192u + sw128_offset(i, ch & 7);
+    *reinterpret_cast<__nv_bfloat16*>(region(base + off)) = __float2bfloat16_rn(v[q]);
   }
 }
 
@@ -106,9 +127,17 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int cj = blockIdx.x;
   const int s = cj / p.HV, j = cj % p.HV;
   const int jq = j / (p.HV / p.HK);
-  const int L = p.chunk_len[s];
+  int L, tok0;
+  if (p.chunk_len) {
+    L = p.chunk_len[s];
+    tok0 = p.chunk_tok0[s];
+  } else {
+    const int c = s % p.cps;
+    tok0 = (s / p.cps) * p.T_row + c * kChunk;
+    L = min(kChunk, p.T_row - c * kChunk);
+  }
   if (L <= 0) return;                                    // unused chunk slot (uniform for the CTA)
-  const int tok0 = p.chunk_tok0[s];
+  HA_PROF(prep, 0);
 
   if (tid == 0) {
     mbar_init(bar_load, 1);
@@ -117,13 +146,15 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     mbar_fence_init();
     prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
   }
-  if (warp == 0) tmem_alloc(tmem_slot, 256);
+  if (warp == 0) tmem_alloc(tmem_slot, 128);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t TM_S = tmem, TM_W = tmem + 64, TM_U = tmem + 128, TM_Q = tmem, TM_O = tmem + 192;
-  const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+  const int rowq = (warp & 3) * 32 + lane;               // accumulator row owned by this thread
+  const int hf = warp >> 2;                              // which 32 of the 64 columns
+  const uint32_t my_tmem = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + hf * 32;
+  HA_PROF(prep, 1);
 
   if (tid == 0) {
     mbar_expect_tx(bar_load, 6 * 8192);
@@ -159,111 +190,146 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   // ---- op #2 KKT (+ Q K^T): S[0:64] = K K^T, S[64:128] = Q K^T
   if (tid == 0) {
+    HA_PROF(prep, 2);
     mbar_wait(bar_load, 0, abort_flag);
+    HA_PROF(prep, 3);
     tc_fence_after_sync();
     const uint32_t id = idesc_bf16(128, 64, false, false);
     const uint32_t base = smem_u32(sm + OFF_KQ);
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       const uint32_t a = base + (ks >> 2) * 16384 + (ks & 3) * 32;
-      umma_ss(TM_S, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(a, 16, 1024, kSwizzle128B), id, ks > 0);
+      umma_ss(tmem, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(a, 16, 1024, kSwizzle128B), id, ks > 0);
     }
     umma_commit(bar_mma);
   }
   __syncthreads();                                       // sEG / sBE visible to everyone
   mbar_wait(bar_mma, 0, abort_flag);
+  HA_PROF(prep, 4);
   tc_fence_after_sync();
   {
-    float v[64];
-    ld64(TM_S + lane_base, v);
-    if (tid < 64) {                                      // row i of A (strictly lower, beta-scaled), fp32
-      const int i = tid;
-      const float gi = sG[i], bi = sBeta[i];
+    float v[32];
+    ld32(my_tmem, v);
+    const int i = rowq & 63;
+    const float gi = sG[i];
+    if (rowq < 64) {                                     // row i of A (strictly lower, beta-scaled), fp32
+      const float bi = sBeta[i];
 #pragma unroll
-      for (int jj = 0; jj < 64; ++jj) {
-        const float e = __expf(fminf(gi - sG[jj], 0.f));
-        sA[i * LDF + jj] = jj < i ? bi * e * v[jj] : 0.f;
+      for (int q = 0; q < 32; ++q) {
+        const int jj = hf * 32 + q;
+        const float e = __expf(gi - sG[jj]);   // <= 0 wherever the entry is kept
+        v[q] = jj < i ? bi * e * v[q] : 0.f;
       }
+#pragma unroll
+      for (int q = 0; q < 32; q += 4)
+        *reinterpret_cast<float4*>(sA + i * LDF + hf * 32 + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
     } else {                                             // row i of P (lower incl. diagonal), bf16 operand tile
-      const int i = tid - 64;
-      const float gi = sG[i];
 #pragma unroll
-      for (int jj = 0; jj < 64; ++jj) {
-        const float e = __expf(fminf(gi - sG[jj], 0.f));
-        v[jj] = jj <= i ? e * v[jj] : 0.f;
+      for (int q = 0; q < 32; ++q) {
+        const int jj = hf * 32 + q;
+        const float e = __expf(gi - sG[jj]);   // <= 0 wherever the entry is kept
+        v[q] = jj <= i ? e * v[q] : 0.f;
       }
-      store_row_image(v, i, sm + OFF_P, nullptr);
+      store_half_row(v, i, hf, sm + OFF_P);
     }
   }
   __syncthreads();
+  HA_PROF(prep, 5);
 
   // ---- op #3 Solve: T = (I + A)^-1, fp32
-  if (warp < 2) {
-    // diagonal 32x32 block `warp`: thread = column, forward substitution down the rows
-    const int o = 32 * warp, c = lane;
-    float x[32];
+  if (tid < 64) {
+    // four 16x16 diagonal blocks; thread = (block, column).  Column-oriented substitution: once x_r is
+    // final, every later row is updated independently (short dependency chain).
+    const int o = (tid >> 4) * 16, c = tid & 15;
+    float y[16];
 #pragma unroll
-    for (int r = 0; r < 32; ++r) {
-      float acc = r == c ? 1.f : 0.f;
-      const float* arow = sA + (o + r) * LDF + o;
+    for (int r = 0; r < 16; ++r) y[r] = r == c ? 1.f : 0.f;
 #pragma unroll
-      for (int jj = 0; jj < r; ++jj) acc = fmaf(-arow[jj], x[jj], acc);
-      x[r] = acc;
-      sT[(o + r) * LDF + o + c] = acc;
+    for (int r = 0; r < 16; ++r) {
+      const float xr = y[r];
+      sT[(o + r) * LDF + o + c] = xr;
+#pragma unroll
+      for (int q = r + 1; q < 16; ++q) y[q] = fmaf(-sA[(o + q) * LDF + o + r], xr, y[q]);
     }
   } else {
-    // upper-right 32x32 block of T is zero
-    const int t2 = tid - 64;
-    for (int idx = t2; idx < 32 * 32; idx += 64) sT[(idx >> 5) * LDF + 32 + (idx & 31)] = 0.f;
+    // blocks above the diagonal are zero: 6 blocks of 16x16
+    for (int idx = tid - 64; idx < 6 * 256; idx += kPrepThreads - 64) {
+      const int blk = idx >> 8, e = idx & 255;
+      const int bi = blk < 3 ? 0 : (blk < 5 ? 1 : 2);
+      const int bj = blk < 3 ? blk + 1 : (blk < 5 ? blk - 1 : 3);
+      sT[(bi * 16 + (e >> 4)) * LDF + bj * 16 + (e & 15)] = 0.f;
+    }
+  }
+  __syncthreads();
+  HA_PROF(prep, 6);
+  {
+    // level 1: blocks (1,0) and (3,2).  X = A_lo T_lo' ; thread -> pair, row, two columns
+    const int pr = tid >> 7, r = (tid & 127) >> 3, c0 = (tid & 7) * 2;
+    const int lo = pr * 32, hi = lo + 16;
+    float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+      const float a = sA[(hi + r) * LDF + lo + m];
+      const float2 t = *reinterpret_cast<const float2*>(sT + (lo + m) * LDF + lo + c0);
+      a0 = fmaf(a, t.x, a0);
+      a1 = fmaf(a, t.y, a1);
+    }
+    sX[(pr * 16 + r) * LDX + c0] = a0;
+    sX[(pr * 16 + r) * LDX + c0 + 1] = a1;
   }
   __syncthreads();
   {
-    // X = A_10 T_00 ; thread -> row r, 8 columns
-    const int r = tid >> 2, c0 = (tid & 3) * 8;
-    float acc[8];
+    const int pr = tid >> 7, r = (tid & 127) >> 3, c0 = (tid & 7) * 2;
+    const int lo = pr * 32, hi = lo + 16;
+    float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-    for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+    for (int m = 0; m < 16; ++m) {
+      const float a = -sT[(hi + r) * LDF + hi + m];      // zero for m > r
+      const float2 x = *reinterpret_cast<const float2*>(sX + (pr * 16 + m) * LDX + c0);
+      a0 = fmaf(a, x.x, a0);
+      a1 = fmaf(a, x.y, a1);
+    }
+    sT[(hi + r) * LDF + lo + c0] = a0;
+    sT[(hi + r) * LDF + lo + c0 + 1] = a1;
+  }
+  __syncthreads();
+  HA_PROF(prep, 7);
+  {
+    // level 2: the 32x32 block (rows 32..63, columns 0..31).  X = A_10 T_00 ; thread -> row, four columns
+    const int r = tid >> 3, c0 = (tid & 7) * 4;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 8
     for (int m = 0; m < 32; ++m) {
       const float a = sA[(32 + r) * LDF + m];
-      const float4 t0 = *reinterpret_cast<const float4*>(sT + m * LDF + c0);
-      const float4 t1 = *reinterpret_cast<const float4*>(sT + m * LDF + c0 + 4);
-      acc[0] = fmaf(a, t0.x, acc[0]); acc[1] = fmaf(a, t0.y, acc[1]);
-      acc[2] = fmaf(a, t0.z, acc[2]); acc[3] = fmaf(a, t0.w, acc[3]);
-      acc[4] = fmaf(a, t1.x, acc[4]); acc[5] = fmaf(a, t1.y, acc[5]);
-      acc[6] = fmaf(a, t1.z, acc[6]); acc[7] = fmaf(a, t1.w, acc[7]);
+      const float4 t = *reinterpret_cast<const float4*>(sT + m * LDF + c0);
+      acc[0] = fmaf(a, t.x, acc[0]); acc[1] = fmaf(a, t.y, acc[1]);
+      acc[2] = fmaf(a, t.z, acc[2]); acc[3] = fmaf(a, t.w, acc[3]);
     }
-#pragma unroll
-    for (int q = 0; q < 8; ++q) sX[r * LDX + c0 + q] = acc[q];
+    *reinterpret_cast<float4*>(sX + r * LDX + c0) = make_float4(acc[0], acc[1], acc[2], acc[3]);
   }
   __syncthreads();
   {
     // T_10 = -T_11 X
-    const int r = tid >> 2, c0 = (tid & 3) * 8;
-    float acc[8];
-#pragma unroll
-    for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+    const int r = tid >> 3, c0 = (tid & 7) * 4;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 8
     for (int m = 0; m < 32; ++m) {
       const float a = -sT[(32 + r) * LDF + 32 + m];      // zero for m > r
-      const float4 x0 = *reinterpret_cast<const float4*>(sX + m * LDX + c0);
-      const float4 x1 = *reinterpret_cast<const float4*>(sX + m * LDX + c0 + 4);
-      acc[0] = fmaf(a, x0.x, acc[0]); acc[1] = fmaf(a, x0.y, acc[1]);
-      acc[2] = fmaf(a, x0.z, acc[2]); acc[3] = fmaf(a, x0.w, acc[3]);
-      acc[4] = fmaf(a, x1.x, acc[4]); acc[5] = fmaf(a, x1.y, acc[5]);
-      acc[6] = fmaf(a, x1.z, acc[6]); acc[7] = fmaf(a, x1.w, acc[7]);
+      const float4 x = *reinterpret_cast<const float4*>(sX + m * LDX + c0);
+      acc[0] = fmaf(a, x.x, acc[0]); acc[1] = fmaf(a, x.y, acc[1]);
+      acc[2] = fmaf(a, x.z, acc[2]); acc[3] = fmaf(a, x.w, acc[3]);
     }
-#pragma unroll
-    for (int q = 0; q < 8; ++q) sT[(32 + r) * LDF + c0 + q] = acc[q];
+    *reinterpret_cast<float4*>(sT + (32 + r) * LDF + c0) = make_float4(acc[0], acc[1], acc[2], acc[3]);
   }
   __syncthreads();
+  HA_PROF(prep, 8);
 
   // ---- column-scaled copies of T as bf16 operand tiles: T^W = T diag(beta e^G), T^U = T diag(beta)
   {
-    const int i = tid >> 1, hf = tid & 1;
+    const int i = tid >> 2, q4 = tid & 3;                // row, quarter (16 columns = two 16-byte pieces)
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int ch = hf * 4 + q;
+    for (int q = 0; q < 2; ++q) {
+      const int ch = q4 * 2 + q;
       float tw[8], tu[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
@@ -283,6 +349,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
+  HA_PROF(prep, 9);
 
   // ---- op #4 W/U: W^T = K^T (T^W)^T, U^T = V^T (T^U)^T  (A operands feature-major straight from the TMA tiles)
   if (tid == 0) {
@@ -290,77 +357,101 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const uint32_t id = idesc_bf16(128, 64, true, false);
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks)
-      umma_ss(TM_W, smem_desc(smem_u32(sm + OFF_KQ) + ks * 2048, 16384, 1024, kSwizzle128B),
+      umma_ss(tmem, smem_desc(smem_u32(sm + OFF_KQ) + ks * 2048, 16384, 1024, kSwizzle128B),
               smem_desc(smem_u32(sm + OFF_TW) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks)
-      umma_ss(TM_U, smem_desc(smem_u32(sm + OFF_V) + ks * 2048, 8192, 1024, kSwizzle128B),
+      umma_ss(tmem + 64, smem_desc(smem_u32(sm + OFF_V) + ks * 2048, 8192, 1024, kSwizzle128B),
               smem_desc(smem_u32(sm + OFF_TU) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
     umma_commit(bar_mma);
   }
   mbar_wait(bar_mma, 1, abort_flag);
+  HA_PROF(prep, 10);
   tc_fence_after_sync();
   {
-    float v[64];
-    ld64(TM_W + lane_base, v);                           // row = key channel tid, columns = tokens
-    store_row_image(v, tid, sm + OFF_WT, p.ws.wq + (size_t)cj * 2 * kImgBytes);
-    ld64(TM_U + lane_base, v);
-    store_row_image(v, tid, sm + OFF_UT, p.ws.u + (size_t)cj * kImgBytes);
+    float v[32];
+    ld32(my_tmem, v);                                    // row = key channel, columns = tokens
+    store_half_row(v, rowq, hf, sm + OFF_WT);
+    ld32(my_tmem + 64, v);
+    store_half_row(v, rowq, hf, sm + OFF_UT);
+    uint8_t* vexp = sm + OFF_V;                          // the V tile is dead: it receives the U export
+    store_token_major(v, rowq, hf, p.nv, [vexp](uint32_t b) { return vexp + b; });
   }
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
+  HA_PROF(prep, 11);
 
-  // ---- chunk-local halves of op #6: (P W)^T = W^T P^T, O_loc^T = U^T P^T
+  // ---- chunk-local halves of op #6: (P W)^T = W^T P^T, O_loc^T = U^T P^T; the W and U images leave meanwhile
   if (tid == 0) {
     tc_fence_after_sync();
     const uint32_t id = idesc_bf16(128, 64, false, false);
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks)
-      umma_ss(TM_Q, smem_desc(smem_u32(sm + OFF_WT) + ks * 32, 16, 1024, kSwizzle128B),
+      umma_ss(tmem, smem_desc(smem_u32(sm + OFF_WT) + ks * 32, 16, 1024, kSwizzle128B),
               smem_desc(smem_u32(sm + OFF_P) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks)
-      umma_ss(TM_O, smem_desc(smem_u32(sm + OFF_UT) + ks * 32, 16, 1024, kSwizzle128B),
+      umma_ss(tmem + 64, smem_desc(smem_u32(sm + OFF_UT) + ks * 32, 16, 1024, kSwizzle128B),
               smem_desc(smem_u32(sm + OFF_P) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
     umma_commit(bar_mma);
+    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes, sm + OFF_WT, kImgBytes);
+    bulk_store(p.ws.u + (size_t)cj * kImgBytes, sm + OFF_V, kImgBytes);
+    bulk_commit();
   }
-  mbar_wait(bar_mma, 0, abort_flag);
-  tc_fence_after_sync();
-  {
-    float v[64];
-    ld64(TM_Q + lane_base, v);
-    // Q~^T[c][i] = Q[i][c] e^{G_i} - (P W)[i][c], c = tid
-    const uint8_t* qtile = sm + OFF_KQ + (tid >> 6) * 16384 + 8192;
-    const int cc = tid & 63;
-#pragma unroll
-    for (int i = 0; i < 64; ++i) {
-      const __nv_bfloat16 qv = *reinterpret_cast<const __nv_bfloat16*>(qtile + sw128_offset(i, cc >> 3) + (cc & 7) * 2);
-      v[i] = fmaf(__bfloat162float(qv), sEG[i], -v[i]);
-    }
-    store_row_image(v, tid, nullptr, p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes);
-    ld64(TM_O + lane_base, v);
-    store_row_image(v, tid, nullptr, p.ws.ol + (size_t)cj * kImgBytes);
-  }
-  {
+  if (tid >= 64) {                                       // per-chunk scalars for the chain kernel
     float* sc = p.ws.sc + (size_t)cj * kScFloats;
     const float gl = sG[63];
-    if (tid < 64) sc[tid] = __expf(gl - sG[tid]);
-    sc[64 + tid] = __expf(gl);
+    const int t = tid - 64;                              // 0..191
+    sc[t] = t < 64 ? __expf(gl - sG[t]) : __expf(gl);
   }
-  if (*abort_flag && tid == 0) report_status(p.status, HA_LA_ERR_TIMEOUT);
+  mbar_wait(bar_mma, 0, abort_flag);
+  HA_PROF(prep, 12);
+  tc_fence_after_sync();
+  {
+    // Q~^T[c][i] = Q[i][c] e^{G_i} - (P W)[i][c], c = rowq; the U^T operand tile is dead and receives the image.
+    float v[32];
+    ld32(my_tmem, v);
+    const uint8_t* qtile = sm + OFF_KQ + (rowq >> 6) * 16384 + 8192;
+    const int cc = rowq & 63;
+#pragma unroll
+    for (int q = 0; q < 32; ++q) {
+      const int i = hf * 32 + q;
+      const __nv_bfloat16 qv = *reinterpret_cast<const __nv_bfloat16*>(qtile + sw128_offset(i, cc >> 3) + (cc & 7) * 2);
+      v[q] = fmaf(__bfloat162float(qv), sEG[i], -v[q]);
+    }
+    store_half_row(v, rowq, hf, sm + OFF_UT);
+    // O_loc export: its two 8 KiB halves go to the two K tiles (both dead)
+    ld32(my_tmem + 64, v);
+    uint8_t* kexp = sm + OFF_KQ;
+    store_token_major(v, rowq, hf, p.nv, [kexp](uint32_t b) { return kexp + (b >> 13) * 16384 + (b & 8191); });
+  }
+  fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, 256);
+  if (tid == 0) {
+    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_UT, kImgBytes);
+    bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_KQ, 8192);
+    bulk_store(p.ws.ol + (size_t)cj * kImgBytes + 8192, sm + OFF_KQ + 16384, 8192);
+    bulk_commit();
+    if (*abort_flag) report_status(p.status, HA_LA_ERR_TIMEOUT);
+  }
+  HA_PROF(prep, 13);
+  if (warp == 0) tmem_dealloc(tmem, 128);
+  if (tid == 0) bulk_wait_read_all();                    // shared memory must outlive the bulk stores' reads
+  HA_PROF(prep, 14);
 }
 
 }  // namespace
 
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream) {
+                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int nv,
+                           cudaStream_t stream) {
   PrepParams pp;
+  pp.nv = nv;
   pp.g = a.g; pp.beta = a.beta;
   pp.chunk_tok0 = plan.chunk_tok0; pp.chunk_len = plan.chunk_len;
+  pp.T_row = p.T_row; pp.cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
   pp.ws = ws; pp.HK = p.HK; pp.HV = p.HV; pp.status = a.status_word;
   const int smem = kPrepSmem + 1024;
   cudaError_t e = cudaFuncSetAttribute(tc_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
