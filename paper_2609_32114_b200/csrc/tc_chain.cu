@@ -39,11 +39,11 @@ constexpr int kChainThreads = 192;       // 4 compute warps + producer warp + MM
 template <int NV> struct ChainCfg {
   static constexpr int kStages = NV == 128 ? 2 : 3;
   static constexpr uint32_t kRowB = NV * 2;                      // bytes of one operand row (NV bf16)
-  static constexpr uint32_t kSliceB = NV * 128;                  // bytes of one 64 x NV export tile
+  static constexpr uint32_t kSliceB = NV * 128;                  // bytes of NV rows of a feature-major image
   static constexpr uint32_t OFF_WQ = 0;                          // 32 KiB
   static constexpr uint32_t OFF_K = 32768;                       // 16 KiB  [kb][64 tok][64 feat]
-  static constexpr uint32_t OFF_U = 49152;                       // 64 x NV tile of U
-  static constexpr uint32_t OFF_O = OFF_U + kSliceB;             // 64 x NV tile of O_loc
+  static constexpr uint32_t OFF_U = 49152;                       // NV rows of the U image
+  static constexpr uint32_t OFF_O = OFF_U + kSliceB;             // NV rows of the O_loc image
   static constexpr uint32_t OFF_SC = OFF_O + kSliceB;            // 192 floats
   static constexpr uint32_t kStageB = (OFF_SC + 768 + 1023) / 1024 * 1024;
   static constexpr uint32_t kTxBytes = 32768 + 16384 + 2 * kSliceB + 768;
@@ -94,18 +94,14 @@ __device__ __forceinline__ void store_brow32(uint8_t* tile, int row, int c0, con
     *reinterpret_cast<uint4*>(tile + brow_offset<NV, ROWS>(row, (c0 >> 3) + q)) = w;
   }
 }
-template <int NV, int ROWS>
-__device__ __forceinline__ void load_brow32(const uint8_t* tile, int row, int c0, float (&v)[32]) {
+// 32 value channels [c0, c0+32) of token `i` from a slice of a feature-major image (row = channel,
+// 128 swizzled bytes = 64 tokens).  Two-byte loads; a warp reads 64 contiguous bytes per channel.
+__device__ __forceinline__ void load_img32(const uint8_t* slice, int i, int c0, float (&v)[32]) {
+  const uint8_t* base = slice + (i & 7) * 2;
+  const int ch = i >> 3;
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const uint4 w = *reinterpret_cast<const uint4*>(tile + brow_offset<NV, ROWS>(row, (c0 >> 3) + q));
-    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      v[q * 8 + 2 * e] = __uint_as_float(u[e] << 16);
-      v[q * 8 + 2 * e + 1] = __uint_as_float(u[e] & 0xffff0000u);
-    }
-  }
+  for (int q = 0; q < 32; ++q)
+    v[q] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(base + sw128_offset(c0 + q, ch)));
 }
 
 __device__ __forceinline__ void ld32f(uint32_t taddr, float (&v)[32]) {
@@ -254,7 +250,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
       const float dec = sc[i];
       const float gam = sc[64 + tid];
       float pre[32];
-      load_brow32<NV, 64>(stage + (tid < 64 ? Cfg::OFF_U : Cfg::OFF_O), i, 0, pre);
+      load_img32(stage + (tid < 64 ? Cfg::OFF_U : Cfg::OFF_O), i, 0, pre);
 
       mbar_wait(bar_mma1, ph, abort_flag);
       HA_PROF(chain, 8 * c + 2);
@@ -264,7 +260,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
         for (int c0 = 0; c0 < NV; c0 += 32) {
           float d[32];
           ld32f(TM1 + lane_base + c0, d);
-          if (c0 > 0) load_brow32<NV, 64>(stage + Cfg::OFF_U, i, c0, pre);
+          if (c0 > 0) load_img32(stage + Cfg::OFF_U, i, c0, pre);
 #pragma unroll
           for (int q = 0; q < 32; ++q) d[q] = (pre[q] - d[q]) * dec;
           store_brow32<NV, 64>(sUt, i, c0, d);
@@ -280,7 +276,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
         for (int c0 = 0; c0 < NV; c0 += 32) {
           float d[32];
           ld32f(TM1 + lane_base + c0, d);
-          if (c0 > 0) load_brow32<NV, 64>(stage + Cfg::OFF_O, i, c0, pre);
+          if (c0 > 0) load_img32(stage + Cfg::OFF_O, i, c0, pre);
 #pragma unroll
           for (int q = 0; q < 32; ++q) d[q] = p.scale * (pre[q] + d[q]);
           if (i < L) {

@@ -2,17 +2,13 @@
 //
 // For every (chunk slot s, V-head j), cj = s * HV + j, the prep kernel writes
 //   wq  [cj] : 32 KiB  W image (16 KiB) followed by the Q~ image (16 KiB)
-//   u   [cj] : 16 KiB  U, token-major export (below)
-//   ol  [cj] : 16 KiB  O_loc, token-major export
+//   u   [cj] : 16 KiB  U image
+//   ol  [cj] : 16 KiB  O_loc image
 //   sc  [cj] : 192 floats  e^{G_L - G_i} for the 64 tokens, then e^{G_L} for the 128 key channels
 // An "image" is a 128 x 64 bf16 matrix stored feature-major: row r (key or value channel) holds the
 // 64 tokens of the chunk in 128 bytes, and the eight 16-byte pieces of a row are stored at piece
 // index (p XOR (r mod 8)).  That is byte for byte the 128-byte-swizzled shared-memory layout that
 // tcgen05.mma reads, so the chain kernel fetches images with plain 1-D bulk copies.
-// A "token-major export" serves the chain kernel's per-token epilogue: for each slice of NV value
-// channels (NV = channels per chain CTA) a contiguous 64 x NV bf16 tile, row = token, stored in the
-// same swizzled row layout the chain kernel uses for its own 64-row MMA operand (64-byte rows and
-// swizzle for NV = 32; 128-byte rows and swizzle, 64 channels per 8 KiB block, otherwise).
 #pragma once
 
 #include "common.cuh"

@@ -10,6 +10,7 @@
 //   #4 W/U    W^T = K^T (T diag(beta e^G))^T,  U^T = V^T (T diag(beta))^T   (M = feature dim = 128)
 // and the chunk-local halves of operator #6, so that the sequential kernel needs one stacked MMA:
 //             Q~ = Q e^G - P W      O_loc = P U        (o = scale [Q~ h + O_loc])
+// (Q e^G enters the Q~ accumulator as one more MMA, Q^T diag(e^G), and P W with the negate-A flag.)
 // Operands arrive by TMA (bf16, 128-byte swizzle), accumulators live in tensor memory, results are
 // assembled in shared memory as ready-to-use operand images (tc_common.cuh) and leave by bulk copy.
 //
@@ -47,6 +48,8 @@ constexpr uint32_t OFF_TW = OFF_R1;                      // bf16 [64][64] K-majo
 constexpr uint32_t OFF_TU = OFF_R1 + 8192;
 constexpr uint32_t OFF_WT = OFF_R1;                      // bf16 [128][64] K-major, swizzled (16 KiB)
 constexpr uint32_t OFF_UT = OFF_R1 + 16384;
+constexpr uint32_t OFF_E = OFF_R1 + 32768;               // bf16 [64][64] diag(e^G), K-major, swizzled; overlaps T's tail and X,
+                                                         // so it is written only after the solve's results were consumed
 constexpr uint32_t OFF_P = OFF_R1 + 40960;               // bf16 [64][64] K-major, swizzled
 constexpr uint32_t OFF_MISC = OFF_P + 8192;              // floats: G[64], beta[64], e^G[64], beta e^G[64]
 constexpr uint32_t OFF_BAR = OFF_MISC + 4 * 64 * 4;
@@ -62,7 +65,6 @@ struct PrepParams {
   int T_row, cps;
   TcWorkspace ws;
   int HK, HV;
-  int nv;                 // value channels per chain CTA (32, 64 or 128): layout of the U / O_loc exports
   int32_t* status;
 };
 
@@ -84,23 +86,6 @@ __device__ __forceinline__ void store_half_row(const float (&v)[32], int row, in
     w.z = pack_bf16(v[q * 8 + 4], v[q * 8 + 5]);
     w.w = pack_bf16(v[q * 8 + 6], v[q * 8 + 7]);
     *reinterpret_cast<uint4*>(tile + sw128_offset(row, hf * 4 + q)) = w;
-  }
-}
-
-// Scatter 32 token values of feature row `r` (tokens 32*hf .. +31) into a token-major export: for each slice
-// of `nv` value channels a 64 x nv bf16 tile in the chain kernel's row layout (64-byte rows with the 64-byte
-// swizzle for nv = 32, else 128-byte rows with the 128-byte swizzle, 64 channels per 8 KiB block).
-// `region(b)` maps export byte b to shared memory.
-template <typename Region>
-__device__ __forceinline__ void store_token_major(const float (&v)[32], int r, int hf, int nv, Region region) {
-  const int slice = r / nv, col = r % nv;
-  const uint32_t base = static_cast<uint32_t>(slice) * nv * 128 + (col & 7) * 2;
-  const int ch = col >> 3;
-#pragma unroll
-  for (int q = 0; q < 32; ++q) {
-    const int i = hf * 32 + q;
-    const uint32_t off = nv == 32 ? sw64_offset(i, ch) : static_cast<uint32_t>(ch >> 3) * 8192u + sw128_offset(i, ch & 7);
-    *reinterpret_cast<__nv_bfloat16*>(region(base + off)) = __float2bfloat16_rn(v[q]);
   }
 }
 
@@ -374,8 +359,19 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     store_half_row(v, rowq, hf, sm + OFF_WT);
     ld32(my_tmem + 64, v);
     store_half_row(v, rowq, hf, sm + OFF_UT);
-    uint8_t* vexp = sm + OFF_V;                          // the V tile is dead: it receives the U export
-    store_token_major(v, rowq, hf, p.nv, [vexp](uint32_t b) { return vexp + b; });
+    // E = diag(e^G) as an MMA operand: Q^T E puts (Q e^G)^T into the accumulator of the Q~ product.
+    // It lies over the tail of the fp32 T matrix, which is dead only now.
+    const int i = tid >> 2;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int ch = (tid & 3) * 2 + q;
+      uint32_t ev[4] = {0u, 0u, 0u, 0u};
+      if ((i >> 3) == ch) {
+        const uint32_t bits = static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(sEG[i])));
+        ev[(i & 7) >> 1] = (i & 1) ? (bits << 16) : bits;
+      }
+      *reinterpret_cast<uint4*>(sm + OFF_E + sw128_offset(i, ch)) = make_uint4(ev[0], ev[1], ev[2], ev[3]);
+    }
   }
   fence_proxy_async_smem();
   tc_fence_before_sync();
@@ -386,17 +382,23 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (tid == 0) {
     tc_fence_after_sync();
     const uint32_t id = idesc_bf16(128, 64, false, false);
+    const uint32_t id_q = idesc_bf16(128, 64, true, false);          // A = Q tile, feature-major
+    const uint32_t id_neg = id | (1u << 13);                         // negate A: accumulate -W^T P^T
 #pragma unroll
-    for (int ks = 0; ks < 4; ++ks)
+    for (int ks = 0; ks < 4; ++ks)                                    // (Q e^G)^T = Q^T E
+      umma_ss(tmem, smem_desc(smem_u32(sm + OFF_KQ) + 8192 + ks * 2048, 16384, 1024, kSwizzle128B),
+              smem_desc(smem_u32(sm + OFF_E) + ks * 32, 16, 1024, kSwizzle128B), id_q, ks > 0);
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks)                                    // ... - W^T P^T  = Q~^T
       umma_ss(tmem, smem_desc(smem_u32(sm + OFF_WT) + ks * 32, 16, 1024, kSwizzle128B),
-              smem_desc(smem_u32(sm + OFF_P) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
+              smem_desc(smem_u32(sm + OFF_P) + ks * 32, 16, 1024, kSwizzle128B), id_neg, 1u);
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks)
       umma_ss(tmem + 64, smem_desc(smem_u32(sm + OFF_UT) + ks * 32, 16, 1024, kSwizzle128B),
               smem_desc(smem_u32(sm + OFF_P) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
     umma_commit(bar_mma);
     bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes, sm + OFF_WT, kImgBytes);
-    bulk_store(p.ws.u + (size_t)cj * kImgBytes, sm + OFF_V, kImgBytes);
+    bulk_store(p.ws.u + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
     bulk_commit();
   }
   if (tid >= 64) {                                       // per-chunk scalars for the chain kernel
@@ -409,28 +411,19 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   HA_PROF(prep, 12);
   tc_fence_after_sync();
   {
-    // Q~^T[c][i] = Q[i][c] e^{G_i} - (P W)[i][c], c = rowq; the U^T operand tile is dead and receives the image.
+    // Q~^T is complete in the accumulator; the V tile is dead and receives its image.
     float v[32];
     ld32(my_tmem, v);
-    const uint8_t* qtile = sm + OFF_KQ + (rowq >> 6) * 16384 + 8192;
-    const int cc = rowq & 63;
-#pragma unroll
-    for (int q = 0; q < 32; ++q) {
-      const int i = hf * 32 + q;
-      const __nv_bfloat16 qv = *reinterpret_cast<const __nv_bfloat16*>(qtile + sw128_offset(i, cc >> 3) + (cc & 7) * 2);
-      v[q] = fmaf(__bfloat162float(qv), sEG[i], -v[q]);
-    }
-    store_half_row(v, rowq, hf, sm + OFF_UT);
-    // O_loc export: its two 8 KiB halves go to the two K tiles (both dead)
+    store_half_row(v, rowq, hf, sm + OFF_V);
+    // O_loc image: rows 0..63 go to the K tile of feature half 0, rows 64..127 to that of half 1 (both dead)
     ld32(my_tmem + 64, v);
-    uint8_t* kexp = sm + OFF_KQ;
-    store_token_major(v, rowq, hf, p.nv, [kexp](uint32_t b) { return kexp + (b >> 13) * 16384 + (b & 8191); });
+    store_half_row(v, rowq & 63, hf, sm + OFF_KQ + (rowq >> 6) * 16384);
   }
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
   if (tid == 0) {
-    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_UT, kImgBytes);
+    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_V, kImgBytes);
     bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_KQ, 8192);
     bulk_store(p.ws.ol + (size_t)cj * kImgBytes + 8192, sm + OFF_KQ + 16384, 8192);
     bulk_commit();
@@ -448,7 +441,7 @@ cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanVi
                            const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int nv,
                            cudaStream_t stream) {
   PrepParams pp;
-  pp.nv = nv;
+  (void)nv;
   pp.g = a.g; pp.beta = a.beta;
   pp.chunk_tok0 = plan.chunk_tok0; pp.chunk_len = plan.chunk_len;
   pp.T_row = p.T_row; pp.cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
