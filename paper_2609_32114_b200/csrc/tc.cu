@@ -69,10 +69,12 @@ int pick_nv(const Problem& p) {
 }  // namespace
 
 bool tc_supported(const Problem& p) {
-  return p.dtype == HA_LA_BF16 && p.variant == HA_LA_GDN && p.dk == 128 && p.dv == 128;
+  return p.dtype == HA_LA_BF16 && p.dk == 128 && p.dv == 128;
 }
 
-size_t tc_workspace_bytes(const Problem& p) { return tc_ws_bytes_for((size_t)p.max_chunks * p.HV); }
+size_t tc_workspace_bytes(const Problem& p) {
+  return tc_ws_bytes_for((size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
+}
 
 int tc_num_launches(const Problem&) { return 2; }
 
@@ -81,7 +83,7 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   if (!make_map(&mq, a.q, p.T_total, p.HK) || !make_map(&mk, a.k, p.T_total, p.HK) ||
       !make_map(&mv, a.v, p.T_total, p.HV))
     return cudaErrorInvalidValue;
-  const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV);
+  const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
   const int nv = pick_nv(p);
   cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, nv, stream);
   if (e != cudaSuccess) return e;

@@ -122,7 +122,7 @@ __device__ __forceinline__ void named_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
-template <int NV>
+template <int NV, bool KDA>
 __global__ void __launch_bounds__(kChainThreads, 1)
 tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   using Cfg = ChainCfg<NV>;
@@ -178,8 +178,12 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
         bulk_load(stage + Cfg::OFF_U, p.ws.u + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
         bulk_load(stage + Cfg::OFF_O, p.ws.ol + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
         bulk_load(stage + Cfg::OFF_SC, p.ws.sc + cj * kScFloats, 768, &bar_full[st]);
-        tma_load_3d(stage + Cfg::OFF_K, &map_k, &bar_full[st], 0, jq, tok0 + c * kChunk);
-        tma_load_3d(stage + Cfg::OFF_K + 8192, &map_k, &bar_full[st], 64, jq, tok0 + c * kChunk);
+        if constexpr (KDA) {   // K e^{G_L - G} from the prep kernel (per-channel decay cannot be applied to U~ rows)
+          bulk_load(stage + Cfg::OFF_K, p.ws.kd + cj * kImgBytes, 16384, &bar_full[st]);
+        } else {
+          tma_load_3d(stage + Cfg::OFF_K, &map_k, &bar_full[st], 0, jq, tok0 + c * kChunk);
+          tma_load_3d(stage + Cfg::OFF_K + 8192, &map_k, &bar_full[st], 64, jq, tok0 + c * kChunk);
+        }
       }
     }
   } else if (warp == 5) {
@@ -327,9 +331,9 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
 }
 
-template <int NV>
+template <int NV, bool KDA>
 cudaError_t launch_nv(const ChainParams& cp, const CUtensorMap& mk, int grid, cudaStream_t stream) {
-  auto kern = tc_chain_kernel<NV>;
+  auto kern = tc_chain_kernel<NV, KDA>;
   const int smem = ChainCfg<NV>::kSmem + 1024;
   static_assert(ChainCfg<NV>::kSmem + 1024 <= 227 * 1024, "shared memory budget");
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -350,9 +354,14 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   cp.ws = ws; cp.HK = p.HK; cp.HV = p.HV; cp.scale = p.scale; cp.status = a.status_word;
   const int grid = p.N * p.HV * (128 / nv);
   if (grid == 0) return cudaSuccess;
-  if (nv == 32) return launch_nv<32>(cp, mk, grid, stream);
-  if (nv == 64) return launch_nv<64>(cp, mk, grid, stream);
-  return launch_nv<128>(cp, mk, grid, stream);
+  if (p.variant == HA_LA_KDA) {
+    if (nv == 32) return launch_nv<32, true>(cp, mk, grid, stream);
+    if (nv == 64) return launch_nv<64, true>(cp, mk, grid, stream);
+    return launch_nv<128, true>(cp, mk, grid, stream);
+  }
+  if (nv == 32) return launch_nv<32, false>(cp, mk, grid, stream);
+  if (nv == 64) return launch_nv<64, false>(cp, mk, grid, stream);
+  return launch_nv<128, false>(cp, mk, grid, stream);
 }
 
 }  // namespace ha_la

@@ -4,6 +4,7 @@
 //   wq  [cj] : 32 KiB  W image (16 KiB) followed by the Q~ image (16 KiB)
 //   u   [cj] : 16 KiB  U image
 //   ol  [cj] : 16 KiB  O_loc image
+//   kd  [cj] : 16 KiB  KDA only: K e^{G_L - G}, in the shared-memory layout of the TMA K tile
 //   sc  [cj] : 192 floats  e^{G_L - G_i} for the 64 tokens, then e^{G_L} for the 128 key channels
 // An "image" is a 128 x 64 bf16 matrix stored feature-major: row r (key or value channel) holds the
 // 64 tokens of the chunk in 128 bytes, and the eight 16-byte pieces of a row are stored at piece
@@ -22,19 +23,22 @@ struct TcWorkspace {
   uint8_t* wq;
   uint8_t* u;
   uint8_t* ol;
+  uint8_t* kd;      // KDA only
   float* sc;
 };
 
-inline __host__ size_t tc_ws_bytes_for(size_t ncj) {
-  return ncj * (2 * kImgBytes + kImgBytes + kImgBytes) + align_up(ncj * kScFloats * sizeof(float), 1024);
+inline __host__ size_t tc_ws_bytes_for(size_t ncj, bool kda) {
+  return ncj * (2 * kImgBytes + kImgBytes + kImgBytes + (kda ? kImgBytes : 0)) +
+         align_up(ncj * kScFloats * sizeof(float), 1024);
 }
 
-inline __host__ TcWorkspace tc_ws_view(void* base, size_t ncj) {
+inline __host__ TcWorkspace tc_ws_view(void* base, size_t ncj, bool kda) {
   TcWorkspace w;
   uint8_t* b = reinterpret_cast<uint8_t*>(base);
   w.wq = b;                      b += ncj * 2 * kImgBytes;
   w.u = b;                       b += ncj * kImgBytes;
   w.ol = b;                      b += ncj * kImgBytes;
+  w.kd = kda ? b : nullptr;      b += kda ? ncj * kImgBytes : 0;
   w.sc = reinterpret_cast<float*>(b);
   return w;
 }

@@ -54,6 +54,11 @@ constexpr uint32_t OFF_P = OFF_R1 + 40960;               // bf16 [64][64] K-majo
 constexpr uint32_t OFF_MISC = OFF_P + 8192;              // floats: G[64], beta[64], e^G[64], beta e^G[64]
 constexpr uint32_t OFF_BAR = OFF_MISC + 4 * 64 * 4;
 constexpr uint32_t kPrepSmem = OFF_BAR + 64;
+// KDA only: per-channel cumulative log-gate (fp32, times log2 e) and the K e^{G_L - G} operand image
+constexpr int LDG = 132;                                  // row stride (floats) of the 64 x 128 gate matrix
+constexpr uint32_t OFF_G = (kPrepSmem + 1023) / 1024 * 1024;
+constexpr uint32_t OFF_KD = (OFF_G + 64 * LDG * 4 + 1023) / 1024 * 1024;   // [kb][64 tok][64 feat], like the K tile
+constexpr uint32_t kPrepSmemKda = OFF_KD + 16384;
 static_assert(OFF_X + 32 * LDX * 4 <= OFF_P, "solve scratch overlaps P");
 static_assert(OFF_UT + 16384 <= OFF_P, "operand tiles overlap P");
 
@@ -76,6 +81,23 @@ __device__ __forceinline__ void ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ float ex2(float x) {          // 2^x, flushes to zero for very negative x
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void unpack8(const uint4& w, float (&f)[8]) {
+  const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    f[2 * e] = __uint_as_float(u[e] << 16);
+    f[2 * e + 1] = __uint_as_float(u[e] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+  return make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+}
+
 // 32 fp32 values (columns 32*hf .. +31 of one 64-column row) -> four 16-byte pieces of bf16, swizzled
 __device__ __forceinline__ void store_half_row(const float (&v)[32], int row, int hf, uint8_t* tile) {
 #pragma unroll
@@ -89,7 +111,8 @@ __device__ __forceinline__ void store_half_row(const float (&v)[32], int row, in
   }
 }
 
-__global__ void __launch_bounds__(kPrepThreads, 2)
+template <bool KDA>
+__global__ void __launch_bounds__(kPrepThreads, KDA ? 1 : 2)
 tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, PrepParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -150,72 +173,189 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
   }
 
-  // ---- op #1 Gate: inclusive scan of the log-gate over the chunk (threads 0..63)
-  if (tid < 64) {
-    const bool valid = tid < L;
-    float x = valid ? p.g[(size_t)(tok0 + tid) * p.HV + j] : 0.f;
-    const float b = valid ? p.beta[(size_t)(tok0 + tid) * p.HV + j] : 0.f;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const float y = __shfl_up_sync(0xffffffffu, x, o);
-      if (lane >= o) x += y;
+  uint32_t mph = 0;                                      // parity of the next MMA-completion wait
+  if constexpr (KDA) {
+    // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
+    float* sGc = reinterpret_cast<float*>(sm + OFF_G);
+    {
+      const float* gsrc = p.g + ((size_t)tok0 * p.HV + j) * 128;
+      for (int idx = tid; idx < 64 * 128; idx += kPrepThreads) {
+        const int i = idx >> 7, c = idx & 127;
+        sGc[i * LDG + c] = i < L ? gsrc[(size_t)i * p.HV * 128 + c] * 1.4426950408889634f : 0.f;
+      }
+      if (tid < 64) {
+        const float b = tid < L ? p.beta[(size_t)(tok0 + tid) * p.HV + j] : 0.f;
+        sBeta[tid] = b;
+        sBE[tid] = b;                                    // the gate factor lives in the K operand, not in T^W
+        sEG[tid] = 1.f;                                  // and Q is rescaled in place: E = identity
+      }
+      // A and P start as zero (entries above the diagonal are never written)
+      for (int idx = tid; idx < 64 * LDF; idx += kPrepThreads) sA[idx] = 0.f;
+      for (int idx = tid; idx < 512; idx += kPrepThreads) reinterpret_cast<uint4*>(sm + OFF_P)[idx] = make_uint4(0, 0, 0, 0);
     }
-    if (tid == 31) *sTmp = x;
-    sBeta[tid] = b;
-    sG[tid] = x;                                         // warp 1 adds warp 0's total below
-  }
-  __syncthreads();
-  if (tid >= 32 && tid < 64) sG[tid] += *sTmp;
-  __syncthreads();
-  if (tid < 64) {
-    const float e = __expf(sG[tid]);
-    sEG[tid] = e;
-    sBE[tid] = e * sBeta[tid];
-  }
+    __syncthreads();
+    {
+      const int c = tid & 127, r0 = (tid >> 7) * 32;     // two threads per channel, 32 rows each
+      float acc = 0.f;
+      for (int i = 0; i < 32; ++i) { acc += sGc[(r0 + i) * LDG + c]; sGc[(r0 + i) * LDG + c] = acc; }
+    }
+    __syncthreads();
+    if (tid >= 128) {
+      const int c = tid & 127;
+      const float add = sGc[31 * LDG + c];
+      for (int i = 32; i < 64; ++i) sGc[i * LDG + c] += add;
+    }
+    mbar_wait(bar_load, 0, abort_flag);                  // every thread reads the K / Q tiles below
+    __syncthreads();
+    HA_PROF(prep, 4);
 
-  // ---- op #2 KKT (+ Q K^T): S[0:64] = K K^T, S[64:128] = Q K^T
-  if (tid == 0) {
-    HA_PROF(prep, 2);
-    mbar_wait(bar_load, 0, abort_flag);
-    HA_PROF(prep, 3);
-    tc_fence_after_sync();
-    const uint32_t id = idesc_bf16(128, 64, false, false);
-    const uint32_t base = smem_u32(sm + OFF_KQ);
+    // ---- op #2 KKT and the masked Q K^T with per-channel decay, element-wise in fp32:
+    //   A_ij = beta_i sum_c k_ic k_jc 2^(G_ic - G_jc) (j < i),  P_ij = sum_c q_ic k_jc 2^(G_ic - G_jc) (j <= i).
+    // Thread (rs, jl) takes rows rs and 63 - rs (together 65 pairs) and the columns j = jl mod 8.
+    {
+      const int jl = tid & 7, rs = tid >> 3;
+#pragma unroll 1
+      for (int pass = 0; pass < 2; ++pass) {
+        const int i = pass == 0 ? rs : 63 - rs;
+        const int nj = jl <= i ? ((i - jl) >> 3) + 1 : 0;
+        float kk[8], qk[8];
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      const uint32_t a = base + (ks >> 2) * 16384 + (ks & 3) * 32;
-      umma_ss(tmem, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(a, 16, 1024, kSwizzle128B), id, ks > 0);
+        for (int m = 0; m < 8; ++m) { kk[m] = 0.f; qk[m] = 0.f; }
+#pragma unroll 1
+        for (int cc = 0; cc < 16; ++cc) {                // 8 channels per step
+          const uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
+          float kif[8], qif[8], gi[8];
+          unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(i, cc & 7)), kif);
+          unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + sw128_offset(i, cc & 7)), qif);
+          *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
+          *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
+#pragma unroll
+          for (int m = 0; m < 8; ++m) {
+            if (m < nj) {
+              const int jj = jl + 8 * m;
+              float kjf[8], gj[8];
+              unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(jj, cc & 7)), kjf);
+              *reinterpret_cast<float4*>(gj) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8);
+              *reinterpret_cast<float4*>(gj + 4) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8 + 4);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float t = kjf[e] * ex2(gi[e] - gj[e]);
+                kk[m] = fmaf(kif[e], t, kk[m]);
+                qk[m] = fmaf(qif[e], t, qk[m]);
+              }
+            }
+          }
+        }
+        const float bi = sBeta[i];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          if (m < nj) {
+            const int jj = jl + 8 * m;
+            if (jj < i) sA[i * LDF + jj] = bi * kk[m];
+            *reinterpret_cast<__nv_bfloat16*>(sm + OFF_P + sw128_offset(i, jj >> 3) + (jj & 7) * 2) =
+                __float2bfloat16_rn(qk[m]);
+          }
+        }
+      }
     }
-    umma_commit(bar_mma);
-  }
-  __syncthreads();                                       // sEG / sBE visible to everyone
-  mbar_wait(bar_mma, 0, abort_flag);
-  HA_PROF(prep, 4);
-  tc_fence_after_sync();
-  {
-    float v[32];
-    ld32(my_tmem, v);
-    const int i = rowq & 63;
-    const float gi = sG[i];
-    if (rowq < 64) {                                     // row i of A (strictly lower, beta-scaled), fp32
-      const float bi = sBeta[i];
+    __syncthreads();                                     // everyone is done with the raw K and Q tiles
+
+    // ---- operands rescaled in place: K <- K 2^G (for W), Q <- Q 2^G (for Q~); K e^{G_L - G} for the chain
+    {
+      const int i = tid >> 2;
 #pragma unroll
-      for (int q = 0; q < 32; ++q) {
-        const int jj = hf * 32 + q;
-        const float e = __expf(gi - sG[jj]);   // <= 0 wherever the entry is kept
-        v[q] = jj < i ? bi * e * v[q] : 0.f;
+      for (int q = 0; q < 4; ++q) {
+        const int cc = (tid & 3) * 4 + q;
+        uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
+        const uint32_t off = sw128_offset(i, cc & 7);
+        float kf[8], qf[8], gi[8], gl[8], kd[8];
+        unpack8(*reinterpret_cast<const uint4*>(kt + off), kf);
+        unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + off), qf);
+        *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
+        *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
+        *reinterpret_cast<float4*>(gl) = *reinterpret_cast<const float4*>(sGc + 63 * LDG + cc * 8);
+        *reinterpret_cast<float4*>(gl + 4) = *reinterpret_cast<const float4*>(sGc + 63 * LDG + cc * 8 + 4);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float eg = ex2(gi[e]);
+          kd[e] = kf[e] * ex2(gl[e] - gi[e]);
+          kf[e] *= eg;
+          qf[e] *= eg;
+        }
+        *reinterpret_cast<uint4*>(kt + off) = pack8(kf);
+        *reinterpret_cast<uint4*>(kt + 8192 + off) = pack8(qf);
+        *reinterpret_cast<uint4*>(sm + OFF_KD + (cc >> 3) * 8192 + off) = pack8(kd);
       }
-#pragma unroll
-      for (int q = 0; q < 32; q += 4)
-        *reinterpret_cast<float4*>(sA + i * LDF + hf * 32 + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
-    } else {                                             // row i of P (lower incl. diagonal), bf16 operand tile
-#pragma unroll
-      for (int q = 0; q < 32; ++q) {
-        const int jj = hf * 32 + q;
-        const float e = __expf(gi - sG[jj]);   // <= 0 wherever the entry is kept
-        v[q] = jj <= i ? e * v[q] : 0.f;
+    }
+  } else {
+    // ---- op #1 Gate: inclusive scan of the log-gate over the chunk (threads 0..63)
+    if (tid < 64) {
+      const bool valid = tid < L;
+      float x = valid ? p.g[(size_t)(tok0 + tid) * p.HV + j] : 0.f;
+      const float b = valid ? p.beta[(size_t)(tok0 + tid) * p.HV + j] : 0.f;
+  #pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += y;
       }
-      store_half_row(v, i, hf, sm + OFF_P);
+      if (tid == 31) *sTmp = x;
+      sBeta[tid] = b;
+      sG[tid] = x;                                         // warp 1 adds warp 0's total below
+    }
+    __syncthreads();
+    if (tid >= 32 && tid < 64) sG[tid] += *sTmp;
+    __syncthreads();
+    if (tid < 64) {
+      const float e = __expf(sG[tid]);
+      sEG[tid] = e;
+      sBE[tid] = e * sBeta[tid];
+    }
+
+    // ---- op #2 KKT (+ Q K^T): S[0:64] = K K^T, S[64:128] = Q K^T
+    if (tid == 0) {
+      HA_PROF(prep, 2);
+      mbar_wait(bar_load, 0, abort_flag);
+      HA_PROF(prep, 3);
+      tc_fence_after_sync();
+      const uint32_t id = idesc_bf16(128, 64, false, false);
+      const uint32_t base = smem_u32(sm + OFF_KQ);
+  #pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t a = base + (ks >> 2) * 16384 + (ks & 3) * 32;
+        umma_ss(tmem, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(a, 16, 1024, kSwizzle128B), id, ks > 0);
+      }
+      umma_commit(bar_mma);
+    }
+    __syncthreads();                                       // sEG / sBE visible to everyone
+    mbar_wait(bar_mma, mph, abort_flag);
+    mph ^= 1;
+    HA_PROF(prep, 4);
+    tc_fence_after_sync();
+    {
+      float v[32];
+      ld32(my_tmem, v);
+      const int i = rowq & 63;
+      const float gi = sG[i];
+      if (rowq < 64) {                                     // row i of A (strictly lower, beta-scaled), fp32
+        const float bi = sBeta[i];
+  #pragma unroll
+        for (int q = 0; q < 32; ++q) {
+          const int jj = hf * 32 + q;
+          const float e = __expf(gi - sG[jj]);   // <= 0 wherever the entry is kept
+          v[q] = jj < i ? bi * e * v[q] : 0.f;
+        }
+  #pragma unroll
+        for (int q = 0; q < 32; q += 4)
+          *reinterpret_cast<float4*>(sA + i * LDF + hf * 32 + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+      } else {                                             // row i of P (lower incl. diagonal), bf16 operand tile
+  #pragma unroll
+        for (int q = 0; q < 32; ++q) {
+          const int jj = hf * 32 + q;
+          const float e = __expf(gi - sG[jj]);   // <= 0 wherever the entry is kept
+          v[q] = jj <= i ? e * v[q] : 0.f;
+        }
+        store_half_row(v, i, hf, sm + OFF_P);
+      }
     }
   }
   __syncthreads();
@@ -350,7 +490,8 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
               smem_desc(smem_u32(sm + OFF_TU) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
     umma_commit(bar_mma);
   }
-  mbar_wait(bar_mma, 1, abort_flag);
+  mbar_wait(bar_mma, mph, abort_flag);
+  mph ^= 1;
   HA_PROF(prep, 10);
   tc_fence_after_sync();
   {
@@ -403,11 +544,16 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
   if (tid >= 64) {                                       // per-chunk scalars for the chain kernel
     float* sc = p.ws.sc + (size_t)cj * kScFloats;
-    const float gl = sG[63];
     const int t = tid - 64;                              // 0..191
-    sc[t] = t < 64 ? __expf(gl - sG[t]) : __expf(gl);
+    if constexpr (KDA) {
+      sc[t] = t < 64 ? 1.f : ex2(reinterpret_cast<const float*>(sm + OFF_G)[63 * LDG + (t - 64)]);
+    } else {
+      const float gl = sG[63];
+      sc[t] = t < 64 ? __expf(gl - sG[t]) : __expf(gl);
+    }
   }
-  mbar_wait(bar_mma, 0, abort_flag);
+  mbar_wait(bar_mma, mph, abort_flag);
+  mph ^= 1;
   HA_PROF(prep, 12);
   tc_fence_after_sync();
   {
@@ -426,6 +572,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_V, kImgBytes);
     bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_KQ, 8192);
     bulk_store(p.ws.ol + (size_t)cj * kImgBytes + 8192, sm + OFF_KQ + 16384, 8192);
+    if constexpr (KDA) bulk_store(p.ws.kd + (size_t)cj * kImgBytes, sm + OFF_KD, kImgBytes);
     bulk_commit();
     if (*abort_flag) report_status(p.status, HA_LA_ERR_TIMEOUT);
   }
@@ -437,6 +584,17 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
 }  // namespace
 
+template <bool KDA>
+static cudaError_t launch_prep_variant(const PrepParams& pp, const CUtensorMap& mq, const CUtensorMap& mk,
+                                       const CUtensorMap& mv, long long grid, cudaStream_t stream) {
+  const int smem = (KDA ? kPrepSmemKda : kPrepSmem) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(tc_prep_kernel<KDA>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  timer_mark(stream, "tc_prep");
+  tc_prep_kernel<KDA><<<(unsigned)grid, kPrepThreads, smem, stream>>>(mq, mk, mv, pp);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                            const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int nv,
                            cudaStream_t stream) {
@@ -446,14 +604,10 @@ cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanVi
   pp.chunk_tok0 = plan.chunk_tok0; pp.chunk_len = plan.chunk_len;
   pp.T_row = p.T_row; pp.cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
   pp.ws = ws; pp.HK = p.HK; pp.HV = p.HV; pp.status = a.status_word;
-  const int smem = kPrepSmem + 1024;
-  cudaError_t e = cudaFuncSetAttribute(tc_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
   const long long grid = (long long)p.max_chunks * p.HV;
   if (grid == 0) return cudaSuccess;
-  timer_mark(stream, "tc_prep");
-  tc_prep_kernel<<<(unsigned)grid, kPrepThreads, smem, stream>>>(mq, mk, mv, pp);
-  return cudaGetLastError();
+  return p.variant == HA_LA_KDA ? launch_prep_variant<true>(pp, mq, mk, mv, grid, stream)
+                                : launch_prep_variant<false>(pp, mq, mk, mv, grid, stream);
 }
 
 }  // namespace ha_la
