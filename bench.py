@@ -131,9 +131,16 @@ def cpu_baseline(inp):
     heads = None
     if est > 25:
         heads = max(cores, int(inp["N"] * w.hv * 20 / est))
-    dt, tokens, threads, desc = oracle_time(inp, heads)
-    return {"value": tokens / dt, "unit": "tokens/s", "cores": threads, "kind": "oracle",
-            "sample": f"{desc}; {dt:.2f} s wall"}
+    # repeat until the sample amounts to roughly 10-30 s of CPU work (cores x wall)
+    total, reps, tokens, threads, desc = 0.0, 0, 0.0, 1, ""
+    while reps < 50:
+        dt, tokens, threads, desc = oracle_time(inp, heads)
+        total += dt
+        reps += 1
+        if total * threads >= 12.0:
+            break
+    return {"value": tokens * reps / total, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+            "sample": f"{desc}; {reps} repetition(s), {total:.2f} s wall in total"}
 
 
 def run_reference(args, inp, rank):
@@ -163,6 +170,27 @@ def run_reference(args, inp, rank):
             "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def rank_seed(rank: int) -> int:
+    """Every rank draws its own batch of the same workload (weak scaling over independent batches)."""
+    return synth.BASE_SEED + 1000 * rank
+
+
+def max_over_ranks(dist, ms: float, device) -> float:
+    """Device-timed milliseconds, maximum over all ranks (the job is as slow as its slowest rank)."""
+    if dist is None:
+        return ms
+    import torch
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world: int, tokens_per_rank: int, ms_per_step: float) -> float:
+    """Whole-job tokens/s: all ranks' tokens over the slowest rank's step time."""
+    return world * tokens_per_rank / (ms_per_step / 1e3)
 
 
 def main():
@@ -201,7 +229,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     # every rank draws its own batch of the same workload (weak scaling over independent batches)
-    inp = synth.make_inputs(w, seed=synth.BASE_SEED + 1000 * rank)
+    inp = synth.make_inputs(w, seed=rank_seed(rank))
     T, N = inp["T"], inp["N"]
     alg_bytes = synth.algorithmic_bytes(w, T, N)
     alg_flops = synth.algorithmic_flops(w, T)
@@ -257,13 +285,9 @@ def main():
     barrier()
     t_wall = time.perf_counter() - t_wall
     step_ms = [a.elapsed_time(b) for a, b in evs]
-    total_ms = float(np.sum(step_ms))
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(dist, float(np.sum(step_ms)), dev)
     ms_per_step = total_ms / args.steps
-    value = world * T / (ms_per_step / 1e3)
+    value = job_throughput(world, T, ms_per_step)
 
     # ---- per-kernel device time (events between kernels), averaged over a few cold-L2 steps
     kt = {}
@@ -281,6 +305,9 @@ def main():
     in_bytes = T * (2 * w.hk * w.dk * e + w.hv * w.dv * e + w.hv * 4 * (1 + (w.dk if w.variant == "kda" else 1)))
     out_bytes = alg_bytes - in_bytes
     kernel_alg_bytes = {"simt_prefill": alg_bytes, "tc_prep": in_bytes, "tc_chain": out_bytes, "plan": 0.0}
+    # DRAM bytes per launch of that kernel from one ncu --set full capture of this workload
+    # (profiles/tc_prep_chain_gdn_layer_4k_ncu_full.md, profiles/tc_prep_chain_kda_8k_ncu_full.md); cold-cache replays
+    ncu_traffic = {("gdn_layer_4k", "tc_chain"): 84.70e6 + 6.58e6, ("gdn_layer_4k", "tc_prep"): 50.92e6 + 18.41e6}
     dom_bytes = kernel_alg_bytes.get(dom, alg_bytes)
     dom_s = kernel_ms[dom] / 1e3
     achieved = dom_bytes / dom_s / 1e9
@@ -288,7 +315,8 @@ def main():
     t_flop = alg_flops / (peaks["bf16_tflops"] * 1e12)
     path_s = ms_per_step / 1e3
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic.get((w.name, dom)),
+                "kernel_alg_bytes": dom_bytes, "peak_source": peaks["source"],
                 "kernel_ms": kernel_ms,
                 "path": {"bound": "hbm" if t_hbm >= t_flop else "tensor", "roofline_us": 1e6 * max(t_hbm, t_flop),
                          "measured_us": 1e6 * path_s, "frac": max(t_hbm, t_flop) / path_s,
@@ -322,12 +350,8 @@ def main():
         e2e_step()
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = {"value": world * T / (e2e_ms / args.steps / 1e3), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
+    e2e_ms = max_over_ranks(dist, e0.elapsed_time(e1), dev)
+    e2e = {"value": job_throughput(world, T, e2e_ms / args.steps), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": int(d2h)}
 
     cpu = None
