@@ -1,16 +1,30 @@
 // Tensor-core (tcgen05) path, host side: tensor maps, workspace carving, slice-width choice, launches.
+//
+// Two launch modes.  Sequential: prep kernel, then chain kernel, both on the caller's stream.
+// Concurrent: the prep kernel runs on an internal stream next to the chain kernel, which
+// consumes each chunk as soon as the prep CTA of that chunk has published it (release/acquire flag
+// per chunk in the workspace, stamped with a per-call epoch so that nothing has to be cleared).  The
+// internal stream forks from and joins back into the caller's stream with two events, so the call
+// stays asynchronous and ordered like any other work on that stream.  The concurrent mode is used
+// when the chain CTAs leave room: NV = 32 (a two-stage chain CTA and a prep CTA fit on one SM
+// together) and at most one chain CTA per two SMs.
 #include <cuda.h>
 #include <stdlib.h>
+
+#include <atomic>
 
 #include "tc_common.cuh"
 
 namespace ha_la {
 
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int nv,
+                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int32_t epoch,
                            cudaStream_t stream);
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                            const CUtensorMap& mk, int nv, cudaStream_t stream);
+                            const CUtensorMap& mk, int nv, int32_t epoch, cudaStream_t stream);
+
+cudaError_t configure_tc_prep(const Problem& p);
+cudaError_t configure_tc_chain(const Problem& p, int nv, bool concurrent);
 
 namespace {
 
@@ -66,6 +80,41 @@ int pick_nv(const Problem& p) {
   return 128;
 }
 
+// Per-device side stream and fork/join events of the concurrent mode, created on first use.
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  bool tried = false, ok = false;
+};
+constexpr int kMaxDevices = 64;
+SideStream g_side[kMaxDevices];
+std::atomic<int32_t> g_epoch{0};
+
+SideStream* side_stream() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  SideStream& s = g_side[dev];
+  if (!s.tried) {
+    s.tried = true;
+    int least = 0, greatest = 0;
+    if (cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess &&
+        cudaStreamCreateWithPriority(&s.stream, cudaStreamNonBlocking, least) == cudaSuccess &&
+        cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) == cudaSuccess &&
+        cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) == cudaSuccess)
+      s.ok = true;
+  }
+  return s.ok ? &s : nullptr;
+}
+
+bool want_concurrent(const Problem& p, int nv) {
+  if (g_timer) return false;                             // per-kernel timing wants one kernel at a time
+  if (const char* e = getenv("HA_LA_TC_OVERLAP")) {
+    if (e[0] == '0') return false;
+  }
+  const long long chain_ctas = (long long)p.N * p.HV * (128 / nv);
+  return nv == 32 && chain_ctas * 2 <= sm_count() && p.max_chunks > 1;
+}
+
 }  // namespace
 
 bool tc_supported(const Problem& p) {
@@ -85,9 +134,34 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
     return cudaErrorInvalidValue;
   const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
   const int nv = pick_nv(p);
-  cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, nv, stream);
+
+  SideStream* side = want_concurrent(p, nv) ? side_stream() : nullptr;
+  // Configure (and load) both kernels before anything is enqueued.
+  cudaError_t ce = configure_tc_prep(p);
+  if (ce != cudaSuccess) return ce;
+  ce = configure_tc_chain(p, nv, side != nullptr);
+  if (ce != cudaSuccess) return ce;
+  if (!side) {
+    cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, 0, stream);
+    if (e != cudaSuccess) return e;
+    return launch_tc_chain(p, a, plan, ws, mk, nv, 0, stream);
+  }
+
+  int32_t epoch = g_epoch.fetch_add(1) + 1;
+  if (epoch == 0) epoch = g_epoch.fetch_add(1) + 1;      // 0 means "sequential"
+  cudaError_t e = cudaEventRecord(side->fork, stream);
   if (e != cudaSuccess) return e;
-  return launch_tc_chain(p, a, plan, ws, mk, nv, stream);
+  e = cudaStreamWaitEvent(side->stream, side->fork, 0);
+  if (e != cudaSuccess) return e;
+  // The chain kernel goes on the caller's stream and is enqueued first, so that its CTAs are resident (one
+  // per SM) before the prep CTAs arrive; the prep kernel runs on the side stream and fills the remaining room.
+  e = launch_tc_chain(p, a, plan, ws, mk, nv, epoch, stream);
+  if (e != cudaSuccess) return e;
+  e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, side->stream);
+  if (e != cudaSuccess) return e;
+  e = cudaEventRecord(side->join, side->stream);
+  if (e != cudaSuccess) return e;
+  return cudaStreamWaitEvent(stream, side->join, 0);
 }
 
 }  // namespace ha_la

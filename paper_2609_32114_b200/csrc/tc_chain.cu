@@ -36,8 +36,8 @@ namespace {
 
 constexpr int kChainThreads = 192;       // 4 compute warps + producer warp + MMA warp
 
-template <int NV> struct ChainCfg {
-  static constexpr int kStages = NV == 128 ? 2 : 3;
+template <int NV, int S_> struct ChainCfg {
+  static constexpr int kStages = S_;
   static constexpr uint32_t kRowB = NV * 2;                      // bytes of one operand row (NV bf16)
   static constexpr uint32_t kSliceB = NV * 128;                  // bytes of NV rows of a feature-major image
   static constexpr uint32_t OFF_WQ = 0;                          // 32 KiB
@@ -65,6 +65,7 @@ struct ChainParams {
   TcWorkspace ws;
   int HK, HV;
   float scale;
+  int32_t epoch;               // != 0: the prep kernel runs concurrently; wait for ws.flags[cj] == epoch per chunk
   int32_t* status;
 };
 
@@ -122,14 +123,13 @@ __device__ __forceinline__ void named_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
-template <int NV, bool KDA>
+template <int NV, bool KDA, int S>
 __global__ void __launch_bounds__(kChainThreads, 1)
 tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
-  using Cfg = ChainCfg<NV>;
-  constexpr int S = Cfg::kStages;
+  using Cfg = ChainCfg<NV, S>;
   constexpr int NSL = 128 / NV;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* sm = smem_raw;                                // no static shared memory in this kernel: 1024-aligned
   uint64_t* bar_full = reinterpret_cast<uint64_t*>(sm + Cfg::OFF_BAR);     // [S]  producer -> everyone
   uint64_t* bar_empty = bar_full + S;                                       // [S]  128 compute threads -> producer
   uint64_t* bar_mma1 = bar_empty + S;                                       // MMA1 complete
@@ -173,6 +173,15 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
         if (c >= S) mbar_wait(&bar_empty[st], ((c / S) - 1) & 1, abort_flag);
         uint8_t* stage = sm + st * Cfg::kStageB;
         const size_t cj = (size_t)(chunk0 + c) * p.HV + j;
+        if (p.epoch != 0) {                              // bounded wait for the prep CTA of this chunk
+          bool ready = false;
+          for (uint32_t it = 0; it < kSpinLimit && !*abort_flag; ++it) {
+            if (ld_acquire_gpu(p.ws.flags + cj) == p.epoch) { ready = true; break; }
+            __nanosleep(40);
+          }
+          if (!ready) *abort_flag = 1;
+          fence_proxy_async_all();
+        }
         mbar_expect_tx(&bar_full[st], Cfg::kTxBytes);
         bulk_load(stage + Cfg::OFF_WQ, p.ws.wq + cj * 2 * kImgBytes, 32768, &bar_full[st]);
         bulk_load(stage + Cfg::OFF_U, p.ws.u + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
@@ -331,37 +340,53 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
 }
 
-template <int NV, bool KDA>
-cudaError_t launch_nv(const ChainParams& cp, const CUtensorMap& mk, int grid, cudaStream_t stream) {
-  auto kern = tc_chain_kernel<NV, KDA>;
-  const int smem = ChainCfg<NV>::kSmem + 1024;
-  static_assert(ChainCfg<NV>::kSmem + 1024 <= 227 * 1024, "shared memory budget");
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
+template <int NV, bool KDA, int S>
+cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, int grid, cudaStream_t stream) {
+  auto kern = tc_chain_kernel<NV, KDA, S>;
+  constexpr int smem = ChainCfg<NV, S>::kSmem;
+  static_assert(smem <= 227 * 1024, "shared memory budget");
+  if (!cp) {                                             // configure only (this also loads the kernel)
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  }
   timer_mark(stream, "tc_chain");
-  kern<<<grid, kChainThreads, smem, stream>>>(mk, cp);
+  kern<<<grid, kChainThreads, smem, stream>>>(*mk, *cp);
   return cudaGetLastError();
+}
+
+template <bool KDA>
+cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, int nv, bool two_stage, int grid,
+                        cudaStream_t stream) {
+  if (nv == 32) return two_stage ? run_nv<32, KDA, 2>(cp, mk, grid, stream) : run_nv<32, KDA, 3>(cp, mk, grid, stream);
+  if (nv == 64) return two_stage ? run_nv<64, KDA, 2>(cp, mk, grid, stream) : run_nv<64, KDA, 3>(cp, mk, grid, stream);
+  return run_nv<128, KDA, 2>(cp, mk, grid, stream);
 }
 
 }  // namespace
 
+// Shared memory of the two-stage NV = 32 chain CTA: with it, one chain CTA and one prep CTA fit on an SM.
+size_t tc_chain_smem_two_stage_nv32() { return ChainCfg<32, 2>::kSmem; }
+
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                            const CUtensorMap& mk, int nv, cudaStream_t stream) {
+                            const CUtensorMap& mk, int nv, int32_t epoch, cudaStream_t stream) {
   ChainParams cp;
   cp.h0 = a.h0; cp.hT = a.hT; cp.o = a.o;
   cp.seq_tok0 = plan.seq_tok0; cp.seq_len = plan.seq_len; cp.seq_chunk0 = plan.seq_chunk0;
   cp.T_row = p.T_row; cp.cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
   cp.ws = ws; cp.HK = p.HK; cp.HV = p.HV; cp.scale = p.scale; cp.status = a.status_word;
+  cp.epoch = epoch;
   const int grid = p.N * p.HV * (128 / nv);
   if (grid == 0) return cudaSuccess;
-  if (p.variant == HA_LA_KDA) {
-    if (nv == 32) return launch_nv<32, true>(cp, mk, grid, stream);
-    if (nv == 64) return launch_nv<64, true>(cp, mk, grid, stream);
-    return launch_nv<128, true>(cp, mk, grid, stream);
-  }
-  if (nv == 32) return launch_nv<32, false>(cp, mk, grid, stream);
-  if (nv == 64) return launch_nv<64, false>(cp, mk, grid, stream);
-  return launch_nv<128, false>(cp, mk, grid, stream);
+  const bool two_stage = epoch != 0;                     // concurrent mode: leave room for a prep CTA on the SM
+  return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, nv, two_stage, grid, stream)
+                                : run_variant<false>(&cp, &mk, nv, two_stage, grid, stream);
+}
+
+// Attributes (and loading) of the chain kernel instance a launch will use; see configure_tc_prep.
+cudaError_t configure_tc_chain(const Problem& p, int nv, bool concurrent) {
+  return p.variant == HA_LA_KDA ? run_variant<true>(nullptr, nullptr, nv, concurrent, 0, nullptr)
+                                : run_variant<false>(nullptr, nullptr, nv, concurrent, 0, nullptr);
 }
 
 }  // namespace ha_la

@@ -51,8 +51,8 @@ constexpr uint32_t OFF_UT = OFF_R1 + 16384;
 constexpr uint32_t OFF_E = OFF_R1 + 32768;               // bf16 [64][64] diag(e^G), K-major, swizzled; overlaps T's tail and X,
                                                          // so it is written only after the solve's results were consumed
 constexpr uint32_t OFF_P = OFF_R1 + 40960;               // bf16 [64][64] K-major, swizzled
-constexpr uint32_t OFF_MISC = OFF_P + 8192;              // floats: G[64], beta[64], e^G[64], beta e^G[64]
-constexpr uint32_t OFF_BAR = OFF_MISC + 4 * 64 * 4;
+constexpr uint32_t OFF_MISC = OFF_P + 8192;              // floats: G[64], beta[64], e^G[64], beta e^G[64], G log2e[64]
+constexpr uint32_t OFF_BAR = OFF_MISC + 5 * 64 * 4;
 constexpr uint32_t kPrepSmem = OFF_BAR + 64;
 // KDA only: per-channel cumulative log-gate (fp32, times log2 e) and the K e^{G_L - G} operand image
 constexpr int LDG = 132;                                  // row stride (floats) of the 64 x 128 gate matrix
@@ -70,6 +70,7 @@ struct PrepParams {
   int T_row, cps;
   TcWorkspace ws;
   int HK, HV;
+  int32_t epoch;          // published to ws.flags[cj] when this CTA's results are in memory (0: do not publish)
   int32_t* status;
 };
 
@@ -98,6 +99,40 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
   return make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
 }
 
+// One warp computes a 16 x 8 tile of C = A B from fp32 matrices in shared memory on the legacy tensor
+// path (mma.sync m16n8k8, TF32) with the 3-term split a = a_hi + a_lo, b = b_hi + b_lo, which keeps the
+// result at fp32 accuracy (the dropped a_lo b_lo term is ~2^-22 relative).  A is row-major (lda), B is
+// row-major K x N (ldb); `ksteps` steps of 8.  Result in the m16n8 accumulator layout:
+// c[0], c[1] = C[g][2t], C[g][2t+1];  c[2], c[3] = C[g+8][2t], C[g+8][2t+1]  (g = lane / 4, t = lane % 4).
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+__device__ __forceinline__ void warp_tile_mm(float (&c)[4], const float* A, int lda, const float* B, int ldb,
+                                             int ksteps, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  c[0] = c[1] = c[2] = c[3] = 0.f;
+  for (int ks = 0; ks < ksteps; ++ks) {
+    const float af[4] = {A[g * lda + ks * 8 + t], A[(g + 8) * lda + ks * 8 + t], A[g * lda + ks * 8 + t + 4],
+                         A[(g + 8) * lda + ks * 8 + t + 4]};
+    const float bf[2] = {B[(ks * 8 + t) * ldb + g], B[(ks * 8 + t + 4) * ldb + g]};
+    uint32_t ah[4], al[4], bh[2], bl[2];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { ah[e] = to_tf32(af[e]); al[e] = to_tf32(af[e] - __uint_as_float(ah[e])); }
+#pragma unroll
+    for (int e = 0; e < 2; ++e) { bh[e] = to_tf32(bf[e]); bl[e] = to_tf32(bf[e] - __uint_as_float(bh[e])); }
+    mma_tf32(c, al, bh);
+    mma_tf32(c, ah, bl);
+    mma_tf32(c, ah, bh);
+  }
+}
+
 // 32 fp32 values (columns 32*hf .. +31 of one 64-column row) -> four 16-byte pieces of bf16, swizzled
 __device__ __forceinline__ void store_half_row(const float (&v)[32], int row, int hf, uint8_t* tile) {
 #pragma unroll
@@ -115,8 +150,8 @@ template <bool KDA>
 __global__ void __launch_bounds__(kPrepThreads, KDA ? 1 : 2)
 tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, PrepParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* sm = smem_raw;                                // no static shared memory in this kernel: 1024-aligned
   float* sA = reinterpret_cast<float*>(sm + OFF_A);
   float* sT = reinterpret_cast<float*>(sm + OFF_T);
   float* sX = reinterpret_cast<float*>(sm + OFF_X);
@@ -145,6 +180,10 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     L = min(kChunk, p.T_row - c * kChunk);
   }
   if (L <= 0) return;                                    // unused chunk slot (uniform for the CTA)
+  if (smem_u32(sm) & 1023u) {                            // the swizzled layouts need it; never seen to fail
+    if (threadIdx.x == 0) report_status(p.status, HA_LA_ERR_DEVICE_CHECK);
+    return;
+  }
   HA_PROF(prep, 0);
 
   if (tid == 0) {
@@ -309,6 +348,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const float e = __expf(sG[tid]);
       sEG[tid] = e;
       sBE[tid] = e * sBeta[tid];
+      sBE[64 + tid] = sG[tid] * 1.4426950408889634f;      // G log2(e), for ex2 in the decay mask
     }
 
     // ---- op #2 KKT (+ Q K^T): S[0:64] = K K^T, S[64:128] = Q K^T
@@ -326,22 +366,23 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       umma_commit(bar_mma);
     }
-    __syncthreads();                                       // sEG / sBE visible to everyone
-    mbar_wait(bar_mma, mph, abort_flag);
+    if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);  // one warp polls; the others sleep at the barrier
     mph ^= 1;
+    __syncthreads();                                     // (also makes sEG / sBE visible to everyone)
     HA_PROF(prep, 4);
     tc_fence_after_sync();
     {
       float v[32];
       ld32(my_tmem, v);
       const int i = rowq & 63;
-      const float gi = sG[i];
+      const float* sG2 = sBE + 64;                       // G log2(e)
+      const float gi = sG2[i];
       if (rowq < 64) {                                     // row i of A (strictly lower, beta-scaled), fp32
         const float bi = sBeta[i];
   #pragma unroll
         for (int q = 0; q < 32; ++q) {
           const int jj = hf * 32 + q;
-          const float e = __expf(gi - sG[jj]);   // <= 0 wherever the entry is kept
+          const float e = ex2(gi - sG2[jj]);     // exponent <= 0 wherever the entry is kept
           v[q] = jj < i ? bi * e * v[q] : 0.f;
         }
   #pragma unroll
@@ -351,7 +392,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   #pragma unroll
         for (int q = 0; q < 32; ++q) {
           const int jj = hf * 32 + q;
-          const float e = __expf(gi - sG[jj]);   // <= 0 wherever the entry is kept
+          const float e = ex2(gi - sG2[jj]);     // exponent <= 0 wherever the entry is kept
           v[q] = jj <= i ? e * v[q] : 0.f;
         }
         store_half_row(v, i, hf, sm + OFF_P);
@@ -388,63 +429,53 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   __syncthreads();
   HA_PROF(prep, 6);
   {
-    // level 1: blocks (1,0) and (3,2).  X = A_lo T_lo' ; thread -> pair, row, two columns
-    const int pr = tid >> 7, r = (tid & 127) >> 3, c0 = (tid & 7) * 2;
-    const int lo = pr * 32, hi = lo + 16;
-    float a0 = 0.f, a1 = 0.f;
-#pragma unroll
-    for (int m = 0; m < 16; ++m) {
-      const float a = sA[(hi + r) * LDF + lo + m];
-      const float2 t = *reinterpret_cast<const float2*>(sT + (lo + m) * LDF + lo + c0);
-      a0 = fmaf(a, t.x, a0);
-      a1 = fmaf(a, t.y, a1);
+    // level 1: blocks (1,0) and (3,2).  X = A_lo T_lo' ; warps 0..3 -> (pair, 8-column tile)
+    if (warp < 4) {
+      const int pr = warp >> 1, nt = warp & 1;
+      const int lo = pr * 32, hi = lo + 16;
+      float c[4];
+      warp_tile_mm(c, sA + hi * LDF + lo, LDF, sT + lo * LDF + lo + nt * 8, LDF, 2, lane);
+      const int g = lane >> 2, t = lane & 3;
+      float* x = sX + (pr * 16) * LDX + nt * 8;
+      x[g * LDX + 2 * t] = c[0]; x[g * LDX + 2 * t + 1] = c[1];
+      x[(g + 8) * LDX + 2 * t] = c[2]; x[(g + 8) * LDX + 2 * t + 1] = c[3];
     }
-    sX[(pr * 16 + r) * LDX + c0] = a0;
-    sX[(pr * 16 + r) * LDX + c0 + 1] = a1;
   }
   __syncthreads();
   {
-    const int pr = tid >> 7, r = (tid & 127) >> 3, c0 = (tid & 7) * 2;
-    const int lo = pr * 32, hi = lo + 16;
-    float a0 = 0.f, a1 = 0.f;
-#pragma unroll
-    for (int m = 0; m < 16; ++m) {
-      const float a = -sT[(hi + r) * LDF + hi + m];      // zero for m > r
-      const float2 x = *reinterpret_cast<const float2*>(sX + (pr * 16 + m) * LDX + c0);
-      a0 = fmaf(a, x.x, a0);
-      a1 = fmaf(a, x.y, a1);
+    if (warp < 4) {                                      // T_lo = -T_hi X
+      const int pr = warp >> 1, nt = warp & 1;
+      const int lo = pr * 32, hi = lo + 16;
+      float c[4];
+      warp_tile_mm(c, sT + hi * LDF + hi, LDF, sX + (pr * 16) * LDX + nt * 8, LDX, 2, lane);
+      const int g = lane >> 2, t = lane & 3;
+      float* d = sT + hi * LDF + lo + nt * 8;
+      d[g * LDF + 2 * t] = -c[0]; d[g * LDF + 2 * t + 1] = -c[1];
+      d[(g + 8) * LDF + 2 * t] = -c[2]; d[(g + 8) * LDF + 2 * t + 1] = -c[3];
     }
-    sT[(hi + r) * LDF + lo + c0] = a0;
-    sT[(hi + r) * LDF + lo + c0 + 1] = a1;
   }
   __syncthreads();
   HA_PROF(prep, 7);
   {
-    // level 2: the 32x32 block (rows 32..63, columns 0..31).  X = A_10 T_00 ; thread -> row, four columns
-    const int r = tid >> 3, c0 = (tid & 7) * 4;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 8
-    for (int m = 0; m < 32; ++m) {
-      const float a = sA[(32 + r) * LDF + m];
-      const float4 t = *reinterpret_cast<const float4*>(sT + m * LDF + c0);
-      acc[0] = fmaf(a, t.x, acc[0]); acc[1] = fmaf(a, t.y, acc[1]);
-      acc[2] = fmaf(a, t.z, acc[2]); acc[3] = fmaf(a, t.w, acc[3]);
-    }
-    *reinterpret_cast<float4*>(sX + r * LDX + c0) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    // level 2: the 32x32 block (rows 32..63, columns 0..31).  X = A_10 T_00 ; warp -> (16-row tile, 8-column tile)
+    const int mt = warp >> 2, nt = warp & 3;
+    float c[4];
+    warp_tile_mm(c, sA + (32 + mt * 16) * LDF, LDF, sT + nt * 8, LDF, 4, lane);
+    const int g = lane >> 2, t = lane & 3;
+    float* x = sX + (mt * 16) * LDX + nt * 8;
+    x[g * LDX + 2 * t] = c[0]; x[g * LDX + 2 * t + 1] = c[1];
+    x[(g + 8) * LDX + 2 * t] = c[2]; x[(g + 8) * LDX + 2 * t + 1] = c[3];
   }
   __syncthreads();
   {
     // T_10 = -T_11 X
-    const int r = tid >> 3, c0 = (tid & 7) * 4;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 8
-    for (int m = 0; m < 32; ++m) {
-      const float a = -sT[(32 + r) * LDF + 32 + m];      // zero for m > r
-      const float4 x = *reinterpret_cast<const float4*>(sX + m * LDX + c0);
-      acc[0] = fmaf(a, x.x, acc[0]); acc[1] = fmaf(a, x.y, acc[1]);
-      acc[2] = fmaf(a, x.z, acc[2]); acc[3] = fmaf(a, x.w, acc[3]);
-    }
-    *reinterpret_cast<float4*>(sT + (32 + r) * LDF + c0) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    const int mt = warp >> 2, nt = warp & 3;
+    float c[4];
+    warp_tile_mm(c, sT + (32 + mt * 16) * LDF + 32, LDF, sX + nt * 8, LDX, 4, lane);
+    const int g = lane >> 2, t = lane & 3;
+    float* d = sT + (32 + mt * 16) * LDF + nt * 8;
+    d[g * LDF + 2 * t] = -c[0]; d[g * LDF + 2 * t + 1] = -c[1];
+    d[(g + 8) * LDF + 2 * t] = -c[2]; d[(g + 8) * LDF + 2 * t + 1] = -c[3];
   }
   __syncthreads();
   HA_PROF(prep, 8);
@@ -490,8 +521,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
               smem_desc(smem_u32(sm + OFF_TU) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
     umma_commit(bar_mma);
   }
-  mbar_wait(bar_mma, mph, abort_flag);
+  if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
   mph ^= 1;
+  __syncthreads();
   HA_PROF(prep, 10);
   tc_fence_after_sync();
   {
@@ -552,8 +584,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       sc[t] = t < 64 ? __expf(gl - sG[t]) : __expf(gl);
     }
   }
-  mbar_wait(bar_mma, mph, abort_flag);
+  if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
   mph ^= 1;
+  __syncthreads();
   HA_PROF(prep, 12);
   tc_fence_after_sync();
   {
@@ -578,28 +611,52 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
   HA_PROF(prep, 13);
   if (warp == 0) tmem_dealloc(tmem, 128);
-  if (tid == 0) bulk_wait_read_all();                    // shared memory must outlive the bulk stores' reads
+  if (tid == 0) {
+    if (p.epoch != 0) {                                  // hand-over to a concurrently running chain kernel
+      bulk_wait_all();
+      fence_proxy_async_all();
+      __threadfence();
+      st_release_gpu(p.ws.flags + cj, p.epoch);
+    } else {
+      bulk_wait_read_all();                              // shared memory must outlive the bulk stores' reads
+    }
+  }
   HA_PROF(prep, 14);
 }
 
 }  // namespace
 
 template <bool KDA>
-static cudaError_t launch_prep_variant(const PrepParams& pp, const CUtensorMap& mq, const CUtensorMap& mk,
-                                       const CUtensorMap& mv, long long grid, cudaStream_t stream) {
-  const int smem = (KDA ? kPrepSmemKda : kPrepSmem) + 1024;
+static cudaError_t configure_prep_variant() {
+  const int smem = KDA ? kPrepSmemKda : kPrepSmem;
   cudaError_t e = cudaFuncSetAttribute(tc_prep_kernel<KDA>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
+  // Same carve-out preference as the chain kernel: kernels that prefer different L1 / shared splits do not
+  // run concurrently, and the two share SMs in the concurrent mode.
+  return cudaFuncSetAttribute(tc_prep_kernel<KDA>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxShared);
+}
+
+template <bool KDA>
+static cudaError_t launch_prep_variant(const PrepParams& pp, const CUtensorMap& mq, const CUtensorMap& mk,
+                                       const CUtensorMap& mv, long long grid, cudaStream_t stream) {
+  const int smem = KDA ? kPrepSmemKda : kPrepSmem;
   timer_mark(stream, "tc_prep");
   tc_prep_kernel<KDA><<<(unsigned)grid, kPrepThreads, smem, stream>>>(mq, mk, mv, pp);
   return cudaGetLastError();
 }
 
+// Sets the kernel's attributes, which also loads it.  Must run before ANY kernel of a concurrent launch is
+// enqueued: loading a kernel for the first time can wait for the device, and the chain kernel would be spinning.
+cudaError_t configure_tc_prep(const Problem& p) {
+  return p.variant == HA_LA_KDA ? configure_prep_variant<true>() : configure_prep_variant<false>();
+}
+
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int nv,
+                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int32_t epoch,
                            cudaStream_t stream) {
   PrepParams pp;
-  (void)nv;
+  pp.epoch = epoch;
   pp.g = a.g; pp.beta = a.beta;
   pp.chunk_tok0 = plan.chunk_tok0; pp.chunk_len = plan.chunk_len;
   pp.T_row = p.T_row; pp.cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
