@@ -11,7 +11,17 @@
   do {                                                                                 \
     if (threadIdx.x == 0 && blockIdx.x == 0 && (slot) < 1024) g_prof_##name[slot] = clock64(); \
   } while (0)
+// records the SM id of CTA `blockIdx.x` at slot base + blockIdx.x % count
+#define HA_PROF_SMID(name, base, count)                                                \
+  do {                                                                                 \
+    if (threadIdx.x == 0) {                                                            \
+      unsigned smid_;                                                                  \
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_));                               \
+      g_prof_##name[(base) + blockIdx.x % (count)] = smid_;                            \
+    }                                                                                  \
+  } while (0)
 #else
+#define HA_PROF_SMID(name, base, count) do { } while (0)
 #define HA_PROF_DECL(name)
 #define HA_PROF(name, slot) do { } while (0)
 #endif

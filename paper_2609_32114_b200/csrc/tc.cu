@@ -19,7 +19,7 @@ namespace ha_la {
 
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                            const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int32_t epoch,
-                           cudaStream_t stream);
+                           int reserved_slots, cudaStream_t stream);
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                             const CUtensorMap& mk, int nv, int32_t epoch, cudaStream_t stream);
 
@@ -112,7 +112,7 @@ bool want_concurrent(const Problem& p, int nv) {
     if (e[0] == '0') return false;
   }
   const long long chain_ctas = (long long)p.N * p.HV * (128 / nv);
-  return nv == 32 && chain_ctas * 2 <= sm_count() && p.max_chunks > 1;
+  return nv <= 64 && chain_ctas * 2 <= sm_count() && p.max_chunks > 1;
 }
 
 }  // namespace
@@ -139,10 +139,10 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   // Configure (and load) both kernels before anything is enqueued.
   cudaError_t ce = configure_tc_prep(p);
   if (ce != cudaSuccess) return ce;
-  ce = configure_tc_chain(p, nv, side != nullptr);
+  ce = configure_tc_chain(p, nv, false);
   if (ce != cudaSuccess) return ce;
   if (!side) {
-    cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, 0, stream);
+    cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, 0, 0, stream);
     if (e != cudaSuccess) return e;
     return launch_tc_chain(p, a, plan, ws, mk, nv, 0, stream);
   }
@@ -157,7 +157,8 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   // per SM) before the prep CTAs arrive; the prep kernel runs on the side stream and fills the remaining room.
   e = launch_tc_chain(p, a, plan, ws, mk, nv, epoch, stream);
   if (e != cudaSuccess) return e;
-  e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, side->stream);
+  // a chain CTA (three stages) fills its SM: the prep kernel gets the other SMs, two CTAs each
+  e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, 2 * p.N * p.HV * (128 / nv), side->stream);
   if (e != cudaSuccess) return e;
   e = cudaEventRecord(side->join, side->stream);
   if (e != cudaSuccess) return e;

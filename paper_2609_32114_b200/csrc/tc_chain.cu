@@ -148,6 +148,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   const int chunk0 = p.seq_tok0 ? p.seq_chunk0[n] : n * p.cps;
   const int nchunks = (len + kChunk - 1) / kChunk;
 
+  HA_PROF_SMID(chain, 768, 128);
   if (tid == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 128); }
     mbar_init(bar_mma1, 1);
@@ -378,7 +379,7 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   cp.epoch = epoch;
   const int grid = p.N * p.HV * (128 / nv);
   if (grid == 0) return cudaSuccess;
-  const bool two_stage = epoch != 0;                     // concurrent mode: leave room for a prep CTA on the SM
+  const bool two_stage = false;                          // three stages also keep prep CTAs off the chain's SMs
   return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, nv, two_stage, grid, stream)
                                 : run_variant<false>(&cp, &mk, nv, two_stage, grid, stream);
 }

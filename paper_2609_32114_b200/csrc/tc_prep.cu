@@ -70,6 +70,7 @@ struct PrepParams {
   int T_row, cps;
   TcWorkspace ws;
   int HK, HV;
+  long long total;        // work items = chunk slots x V-heads
   int32_t epoch;          // published to ws.flags[cj] when this CTA's results are in memory (0: do not publish)
   int32_t* status;
 };
@@ -167,24 +168,12 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
-  const int cj = blockIdx.x;
-  const int s = cj / p.HV, j = cj % p.HV;
-  const int jq = j / (p.HV / p.HK);
-  int L, tok0;
-  if (p.chunk_len) {
-    L = p.chunk_len[s];
-    tok0 = p.chunk_tok0[s];
-  } else {
-    const int c = s % p.cps;
-    tok0 = (s / p.cps) * p.T_row + c * kChunk;
-    L = min(kChunk, p.T_row - c * kChunk);
-  }
-  if (L <= 0) return;                                    // unused chunk slot (uniform for the CTA)
   if (smem_u32(sm) & 1023u) {                            // the swizzled layouts need it; never seen to fail
     if (threadIdx.x == 0) report_status(p.status, HA_LA_ERR_DEVICE_CHECK);
     return;
   }
   HA_PROF(prep, 0);
+  HA_PROF_SMID(prep, 256, 512);
 
   if (tid == 0) {
     mbar_init(bar_load, 1);
@@ -203,6 +192,29 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const uint32_t my_tmem = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + hf * 32;
   HA_PROF(prep, 1);
 
+  // Persistent CTA: work items (chunk slot, V-head) blockIdx.x, blockIdx.x + gridDim.x, ... in that order, so
+  // that early chunks are finished first (the chain kernel may be consuming them concurrently).
+  uint32_t mph = 0;                                      // parity of the next MMA-completion wait
+  uint32_t lph = 0;                                      // parity of the next tile-load wait
+  long long prev_cj = -1;                                // item whose bulk stores are still in flight (thread 0)
+  for (long long cjl = blockIdx.x; cjl < p.total; cjl += gridDim.x) {
+  const size_t cj = (size_t)cjl;
+  const int s = (int)(cjl / p.HV), j = (int)(cjl % p.HV);
+  const int jq = j / (p.HV / p.HK);
+  int L, tok0;
+  if (p.chunk_len) {
+    L = p.chunk_len[s];
+    tok0 = p.chunk_tok0[s];
+  } else {
+    const int c = s % p.cps;
+    tok0 = (s / p.cps) * p.T_row + c * kChunk;
+    L = min(kChunk, p.T_row - c * kChunk);
+  }
+  if (L <= 0) continue;                                  // unused chunk slot (uniform for the CTA)
+
+  // The previous item's bulk stores must have read their shared-memory sources before anything is overwritten.
+  if (tid == 0 && prev_cj >= 0) bulk_wait_read_all();
+  __syncthreads();
   if (tid == 0) {
     mbar_expect_tx(bar_load, 6 * 8192);
     for (int kb = 0; kb < 2; ++kb) {
@@ -210,9 +222,13 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       tma_load_3d(sm + OFF_KQ + kb * 16384 + 8192, &map_q, bar_load, kb * 64, jq, tok0);
       tma_load_3d(sm + OFF_V + kb * 8192, &map_v, bar_load, kb * 64, j, tok0);
     }
+    if (p.epoch != 0 && prev_cj >= 0) {                  // publish the previous item under the cover of these loads
+      bulk_wait_all();
+      fence_proxy_async_all();
+      __threadfence();
+      st_release_gpu(p.ws.flags + prev_cj, p.epoch);
+    }
   }
-
-  uint32_t mph = 0;                                      // parity of the next MMA-completion wait
   if constexpr (KDA) {
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
     float* sGc = reinterpret_cast<float*>(sm + OFF_G);
@@ -244,7 +260,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const float add = sGc[31 * LDG + c];
       for (int i = 32; i < 64; ++i) sGc[i * LDG + c] += add;
     }
-    mbar_wait(bar_load, 0, abort_flag);                  // every thread reads the K / Q tiles below
+    mbar_wait(bar_load, lph, abort_flag);                // every thread reads the K / Q tiles below
     __syncthreads();
     HA_PROF(prep, 4);
 
@@ -354,7 +370,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ---- op #2 KKT (+ Q K^T): S[0:64] = K K^T, S[64:128] = Q K^T
     if (tid == 0) {
       HA_PROF(prep, 2);
-      mbar_wait(bar_load, 0, abort_flag);
+      mbar_wait(bar_load, lph, abort_flag);
       HA_PROF(prep, 3);
       tc_fence_after_sync();
       const uint32_t id = idesc_bf16(128, 64, false, false);
@@ -607,18 +623,25 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     bulk_store(p.ws.ol + (size_t)cj * kImgBytes + 8192, sm + OFF_KQ + 16384, 8192);
     if constexpr (KDA) bulk_store(p.ws.kd + (size_t)cj * kImgBytes, sm + OFF_KD, kImgBytes);
     bulk_commit();
-    if (*abort_flag) report_status(p.status, HA_LA_ERR_TIMEOUT);
+    prev_cj = cjl;
   }
+  lph ^= 1;
   HA_PROF(prep, 13);
+  }  // work items
+
+  __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, 128);
   if (tid == 0) {
-    if (p.epoch != 0) {                                  // hand-over to a concurrently running chain kernel
-      bulk_wait_all();
-      fence_proxy_async_all();
-      __threadfence();
-      st_release_gpu(p.ws.flags + cj, p.epoch);
-    } else {
-      bulk_wait_read_all();                              // shared memory must outlive the bulk stores' reads
+    if (*abort_flag) report_status(p.status, HA_LA_ERR_TIMEOUT);
+    if (prev_cj >= 0) {
+      if (p.epoch != 0) {                                // hand-over to a concurrently running chain kernel
+        bulk_wait_all();
+        fence_proxy_async_all();
+        __threadfence();
+        st_release_gpu(p.ws.flags + prev_cj, p.epoch);
+      } else {
+        bulk_wait_read_all();                            // shared memory must outlive the bulk stores' reads
+      }
     }
   }
   HA_PROF(prep, 14);
@@ -654,15 +677,21 @@ cudaError_t configure_tc_prep(const Problem& p) {
 
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                            const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int32_t epoch,
-                           cudaStream_t stream) {
+                           int reserved_slots, cudaStream_t stream) {
   PrepParams pp;
   pp.epoch = epoch;
   pp.g = a.g; pp.beta = a.beta;
   pp.chunk_tok0 = plan.chunk_tok0; pp.chunk_len = plan.chunk_len;
   pp.T_row = p.T_row; pp.cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
   pp.ws = ws; pp.HK = p.HK; pp.HV = p.HV; pp.status = a.status_word;
-  const long long grid = (long long)p.max_chunks * p.HV;
-  if (grid == 0) return cudaSuccess;
+  pp.total = (long long)p.max_chunks * p.HV;
+  if (pp.total == 0) return cudaSuccess;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  // resident CTAs; in the concurrent mode every chain CTA takes the place of one of them
+  long long slots = (long long)sms * (p.variant == HA_LA_KDA ? 1 : 2) - reserved_slots;
+  if (slots < 1) slots = 1;
+  const long long grid = pp.total < slots ? pp.total : slots;
   return p.variant == HA_LA_KDA ? launch_prep_variant<true>(pp, mq, mk, mv, grid, stream)
                                 : launch_prep_variant<false>(pp, mq, mk, mv, grid, stream);
 }
