@@ -58,7 +58,14 @@ constexpr uint32_t kPrepSmem = OFF_BAR + 64;
 constexpr int LDG = 132;                                  // row stride (floats) of the 64 x 128 gate matrix
 constexpr uint32_t OFF_G = (kPrepSmem + 1023) / 1024 * 1024;
 constexpr uint32_t OFF_KD = (OFF_G + 64 * LDG * 4 + 1023) / 1024 * 1024;   // [kb][64 tok][64 feat], like the K tile
-constexpr uint32_t kPrepSmemKda = OFF_KD + 16384;
+// K+ / Q+ rows (block b: 16 K+ rows then 16 Q+ rows; 160 rows so that an M = 64 operand may start at row 96)
+constexpr uint32_t OFF_KQP = OFF_KD + 16384;              // [kb][160 rows][128 B], K-major, swizzled
+constexpr uint32_t KQP_KB = 160 * 128;
+// K- rows for block-rows I = 1, 2, 3 (16, 32, 48 rows, starting at rows 0, 16, 48)
+constexpr uint32_t OFF_KM = OFF_KQP + 2 * KQP_KB;         // [kb][96 rows][128 B], K-major, swizzled
+constexpr uint32_t KM_KB = 96 * 128;
+constexpr uint32_t kPrepSmemKda = OFF_KM + 2 * KM_KB;
+static_assert(kPrepSmemKda <= 227 * 1024, "KDA shared memory budget");
 static_assert(OFF_X + 32 * LDX * 4 <= OFF_P, "solve scratch overlaps P");
 static_assert(OFF_UT + 16384 <= OFF_P, "operand tiles overlap P");
 
@@ -264,51 +271,128 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     __syncthreads();
     HA_PROF(prep, 4);
 
-    // ---- op #2 KKT and the masked Q K^T with per-channel decay, element-wise in fp32:
+    // ---- op #2 KKT and the masked Q K^T with per-channel decay:
     //   A_ij = beta_i sum_c k_ic k_jc 2^(G_ic - G_jc) (j < i),  P_ij = sum_c q_ic k_jc 2^(G_ic - G_jc) (j <= i).
-    // Thread (rs, jl) takes rows rs and 63 - rs (together 65 pairs) and the columns j = jl mod 8.
+    // Tokens are grouped in blocks of 16.  For i in block I and j in an EARLIER block the decay factors through
+    // the gate R_I at the first token of block I:  2^(G_i - R_I) * 2^(R_I - G_j), both exponents <= 0, so the
+    // off-diagonal blocks are plain contractions of rescaled bf16 operands and go to the tensor cores:
+    //   K+_i = k_i 2^(G_i - R_I), Q+_i = q_i 2^(G_i - R_I)   (one copy),   K-_j^(I) = k_j 2^(R_I - G_j)  (per block-row I).
+    // The four diagonal blocks are evaluated element-wise in fp32.
     {
-      const int jl = tid & 7, rs = tid >> 3;
+      const int i = tid >> 2, bi16 = i >> 4;
+      const int row_k = 32 * bi16 + (i & 15);
 #pragma unroll 1
-      for (int pass = 0; pass < 2; ++pass) {
-        const int i = pass == 0 ? rs : 63 - rs;
-        const int nj = jl <= i ? ((i - jl) >> 3) + 1 : 0;
-        float kk[8], qk[8];
+      for (int q = 0; q < 4; ++q) {
+        const int cc = (tid & 3) * 4 + q;
+        const uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
+        const uint32_t off = sw128_offset(i, cc & 7);
+        float kf[8], qf[8], gi[8], gr[8], t8[8];
+        unpack8(*reinterpret_cast<const uint4*>(kt + off), kf);
+        unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + off), qf);
+        *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
+        *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
+        *reinterpret_cast<float4*>(gr) = *reinterpret_cast<const float4*>(sGc + (bi16 * 16) * LDG + cc * 8);
+        *reinterpret_cast<float4*>(gr + 4) = *reinterpret_cast<const float4*>(sGc + (bi16 * 16) * LDG + cc * 8 + 4);
+        uint8_t* kqp = sm + OFF_KQP + (cc >> 3) * KQP_KB;
 #pragma unroll
-        for (int m = 0; m < 8; ++m) { kk[m] = 0.f; qk[m] = 0.f; }
-#pragma unroll 1
-        for (int cc = 0; cc < 16; ++cc) {                // 8 channels per step
-          const uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
-          float kif[8], qif[8], gi[8];
-          unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(i, cc & 7)), kif);
-          unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + sw128_offset(i, cc & 7)), qif);
-          *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
-          *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
+        for (int e = 0; e < 8; ++e) { gr[e] = ex2(gi[e] - gr[e]); t8[e] = kf[e] * gr[e]; }
+        *reinterpret_cast<uint4*>(kqp + sw128_offset(row_k, cc & 7)) = pack8(t8);
 #pragma unroll
-          for (int m = 0; m < 8; ++m) {
-            if (m < nj) {
-              const int jj = jl + 8 * m;
-              float kjf[8], gj[8];
-              unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(jj, cc & 7)), kjf);
-              *reinterpret_cast<float4*>(gj) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8);
-              *reinterpret_cast<float4*>(gj + 4) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8 + 4);
+        for (int e = 0; e < 8; ++e) t8[e] = qf[e] * gr[e];
+        *reinterpret_cast<uint4*>(kqp + sw128_offset(row_k + 16, cc & 7)) = pack8(t8);
+        for (int I2 = bi16 + 1; I2 < 4; ++I2) {          // K- copies for the later block-rows
+          float g2[8];
+          *reinterpret_cast<float4*>(g2) = *reinterpret_cast<const float4*>(sGc + (I2 * 16) * LDG + cc * 8);
+          *reinterpret_cast<float4*>(g2 + 4) = *reinterpret_cast<const float4*>(sGc + (I2 * 16) * LDG + cc * 8 + 4);
 #pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                const float t = kjf[e] * ex2(gi[e] - gj[e]);
-                kk[m] = fmaf(kif[e], t, kk[m]);
-                qk[m] = fmaf(qif[e], t, qk[m]);
-              }
-            }
-          }
+          for (int e = 0; e < 8; ++e) t8[e] = kf[e] * ex2(g2[e] - gi[e]);
+          const int r0 = I2 == 1 ? 0 : (I2 == 2 ? 16 : 48);
+          *reinterpret_cast<uint4*>(sm + OFF_KM + (cc >> 3) * KM_KB + sw128_offset(r0 + i, cc & 7)) = pack8(t8);
         }
-        const float bi = sBeta[i];
+      }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {                                      // block-row I: D_I[64 x 16 I] = [K+_I ; Q+_I ; ...] (K-^(I))^T
+      tc_fence_after_sync();
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          if (m < nj) {
-            const int jj = jl + 8 * m;
-            if (jj < i) sA[i * LDF + jj] = bi * kk[m];
-            *reinterpret_cast<__nv_bfloat16*>(sm + OFF_P + sw128_offset(i, jj >> 3) + (jj & 7) * 2) =
-                __float2bfloat16_rn(qk[m]);
+      for (int I = 1; I < 4; ++I) {
+        const uint32_t id = idesc_bf16(64, 16 * I, false, false);
+        const uint32_t col = I == 1 ? 0 : (I == 2 ? 16 : 48);
+        const uint32_t r0 = col;                         // first K- row of this block-row = its column offset
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t a = smem_u32(sm + OFF_KQP) + (ks >> 2) * KQP_KB + (32 * I) * 128 + (ks & 3) * 32;
+          const uint32_t bb = smem_u32(sm + OFF_KM) + (ks >> 2) * KM_KB + r0 * 128 + (ks & 3) * 32;
+          umma_ss(tmem + col, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(bb, 16, 1024, kSwizzle128B), id, ks > 0);
+        }
+      }
+      umma_commit(bar_mma);
+    }
+    // diagonal 16x16 blocks, element-wise (overlaps the MMAs): 4 blocks x 136 pairs (j <= i)
+    for (int pidx = tid; pidx < 4 * 136; pidx += kPrepThreads) {
+      const int blk = pidx / 136, qq = pidx % 136;
+      int il = 0;
+      while ((il + 1) * (il + 2) / 2 <= qq) ++il;
+      const int jl = qq - il * (il + 1) / 2;
+      const int i = blk * 16 + il, jj = blk * 16 + jl;
+      float kk = 0.f, qk = 0.f;
+#pragma unroll 2
+      for (int cc = 0; cc < 16; ++cc) {
+        const uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
+        float kif[8], qif[8], kjf[8], gi[8], gj[8];
+        unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(i, cc & 7)), kif);
+        unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + sw128_offset(i, cc & 7)), qif);
+        unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(jj, cc & 7)), kjf);
+        *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
+        *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
+        *reinterpret_cast<float4*>(gj) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8);
+        *reinterpret_cast<float4*>(gj + 4) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8 + 4);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float t = kjf[e] * ex2(gi[e] - gj[e]);
+          kk = fmaf(kif[e], t, kk);
+          qk = fmaf(qif[e], t, qk);
+        }
+      }
+      if (jj < i) sA[i * LDF + jj] = sBeta[i] * kk;
+      *reinterpret_cast<__nv_bfloat16*>(sm + OFF_P + sw128_offset(i, jj >> 3) + (jj & 7) * 2) = __float2bfloat16_rn(qk);
+    }
+    if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
+    mph ^= 1;
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp < 2) {
+      // M = 64 accumulators: row r sits in lane (r % 16) + 32 (r / 16).  Rows 0..15 (K+ -> K K^T) are lanes
+      // 0..15 of warp 0, rows 16..31 (Q+ -> Q K^T) lanes 0..15 of warp 1; the other rows are padding.
+      const uint32_t tl = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+      uint32_t r1[16], r2[32], r3a[32], r3b[16];
+      tmem_ld16(tl + 0, r1);
+      tmem_ld32(tl + 16, r2);
+      tmem_ld32(tl + 48, r3a);
+      tmem_ld16(tl + 80, r3b);
+      tmem_ld_wait();
+      if (lane < 16) {
+#pragma unroll
+        for (int I = 1; I < 4; ++I) {
+          const int i = 16 * I + lane;
+          float v[48];
+#pragma unroll
+          for (int c = 0; c < 16 * I; ++c)
+            v[c] = __uint_as_float(I == 1 ? r1[c] : (I == 2 ? r2[c] : (c < 32 ? r3a[c] : r3b[c - 32])));
+          if (warp == 0) {
+            const float bi = sBeta[i];
+#pragma unroll
+            for (int c = 0; c < 16 * I; c += 4)
+              *reinterpret_cast<float4*>(sA + i * LDF + c) = make_float4(bi * v[c], bi * v[c + 1], bi * v[c + 2], bi * v[c + 3]);
+          } else {
+#pragma unroll
+            for (int ch = 0; ch < 2 * I; ++ch) {
+              const float t8[8] = {v[ch * 8], v[ch * 8 + 1], v[ch * 8 + 2], v[ch * 8 + 3],
+                                   v[ch * 8 + 4], v[ch * 8 + 5], v[ch * 8 + 6], v[ch * 8 + 7]};
+              *reinterpret_cast<uint4*>(sm + OFF_P + sw128_offset(i, ch)) = pack8(t8);
+            }
           }
         }
       }
