@@ -204,38 +204,52 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   uint32_t mph = 0;                                      // parity of the next MMA-completion wait
   uint32_t lph = 0;                                      // parity of the next tile-load wait
   long long prev_cj = -1;                                // item whose bulk stores are still in flight (thread 0)
-  for (long long cjl = blockIdx.x; cjl < p.total; cjl += gridDim.x) {
-  const size_t cj = (size_t)cjl;
-  const int s = (int)(cjl / p.HV), j = (int)(cjl % p.HV);
-  const int jq = j / (p.HV / p.HK);
-  int L, tok0;
-  if (p.chunk_len) {
-    L = p.chunk_len[s];
-    tok0 = p.chunk_tok0[s];
-  } else {
-    const int c = s % p.cps;
-    tok0 = (s / p.cps) * p.T_row + c * kChunk;
-    L = min(kChunk, p.T_row - c * kChunk);
-  }
-  if (L <= 0) continue;                                  // unused chunk slot (uniform for the CTA)
-
-  // The previous item's bulk stores must have read their shared-memory sources before anything is overwritten.
-  if (tid == 0 && prev_cj >= 0) bulk_wait_read_all();
-  __syncthreads();
-  if (tid == 0) {
+  auto item_geom = [&](long long c, int& j_, int& jq_, int& L_, int& tok0_) {
+    const int s_ = (int)(c / p.HV);
+    j_ = (int)(c % p.HV);
+    jq_ = j_ / (p.HV / p.HK);
+    if (p.chunk_len) {
+      L_ = p.chunk_len[s_];
+      tok0_ = p.chunk_tok0[s_];
+    } else {
+      const int cc_ = s_ % p.cps;
+      tok0_ = (s_ / p.cps) * p.T_row + cc_ * kChunk;
+      L_ = min(kChunk, p.T_row - cc_ * kChunk);
+    }
+  };
+  auto issue_tiles = [&](int j_, int jq_, int tok0_) {   // thread 0: K, Q, V tiles of one item
     mbar_expect_tx(bar_load, 6 * 8192);
     for (int kb = 0; kb < 2; ++kb) {
-      tma_load_3d(sm + OFF_KQ + kb * 16384, &map_k, bar_load, kb * 64, jq, tok0);
-      tma_load_3d(sm + OFF_KQ + kb * 16384 + 8192, &map_q, bar_load, kb * 64, jq, tok0);
-      tma_load_3d(sm + OFF_V + kb * 8192, &map_v, bar_load, kb * 64, j, tok0);
+      tma_load_3d(sm + OFF_KQ + kb * 16384, &map_k, bar_load, kb * 64, jq_, tok0_);
+      tma_load_3d(sm + OFF_KQ + kb * 16384 + 8192, &map_q, bar_load, kb * 64, jq_, tok0_);
+      tma_load_3d(sm + OFF_V + kb * 8192, &map_v, bar_load, kb * 64, j_, tok0_);
     }
-    if (p.epoch != 0 && prev_cj >= 0) {                  // publish the previous item under the cover of these loads
+  };
+  auto publish_prev = [&]() {                            // thread 0, concurrent mode: hand the previous item over
+    if (p.epoch != 0 && prev_cj >= 0) {
       bulk_wait_all();
       fence_proxy_async_all();
       __threadfence();
       st_release_gpu(p.ws.flags + prev_cj, p.epoch);
     }
+  };
+  long long cjl = blockIdx.x;
+  int j = 0, jq = 0, L = 0, tok0 = 0;
+  bool have = cjl < p.total;
+  if (have) { item_geom(cjl, j, jq, L, tok0); have = L > 0; }   // unused chunk slots come last
+  float g_pre = 0.f, b_pre = 0.f;                        // GDN, threads 0..63: this token's log-gate and beta
+  if (have) {
+    if (tid == 0) issue_tiles(j, jq, tok0);
+    if (!KDA && tid < L && tid < 64) {
+      g_pre = p.g[(size_t)(tok0 + tid) * p.HV + j];
+      b_pre = p.beta[(size_t)(tok0 + tid) * p.HV + j];
+    }
   }
+  while (have) {
+  const size_t cj = (size_t)cjl;
+  // The previous item's bulk stores must have read their shared-memory sources before anything is overwritten.
+  if (tid == 0 && prev_cj >= 0) bulk_wait_read_all();
+  __syncthreads();
   if constexpr (KDA) {
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
     float* sGc = reinterpret_cast<float*>(sm + OFF_G);
@@ -329,6 +343,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       umma_commit(bar_mma);
+      publish_prev();
     }
     // diagonal 16x16 blocks, element-wise (overlaps the MMAs): 4 blocks x 136 pairs (j <= i)
     for (int pidx = tid; pidx < 4 * 136; pidx += kPrepThreads) {
@@ -429,9 +444,8 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   } else {
     // ---- op #1 Gate: inclusive scan of the log-gate over the chunk (threads 0..63)
     if (tid < 64) {
-      const bool valid = tid < L;
-      float x = valid ? p.g[(size_t)(tok0 + tid) * p.HV + j] : 0.f;
-      const float b = valid ? p.beta[(size_t)(tok0 + tid) * p.HV + j] : 0.f;
+      float x = g_pre;                                   // fetched while the previous item was finishing
+      const float b = b_pre;
   #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         const float y = __shfl_up_sync(0xffffffffu, x, o);
@@ -465,6 +479,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         umma_ss(tmem, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(a, 16, 1024, kSwizzle128B), id, ks > 0);
       }
       umma_commit(bar_mma);
+      publish_prev();
     }
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);  // one warp polls; the others sleep at the barrier
     mph ^= 1;
@@ -685,31 +700,44 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
   }
   if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
+  if (tid == 0) bulk_wait_read_all();                    // the W^T / U^T tiles were read; they receive the next images
   mph ^= 1;
   __syncthreads();
   HA_PROF(prep, 12);
   tc_fence_after_sync();
+  // Every MMA of this item is done, so the K / Q / V tile regions are free: start the next item's loads now.
+  const long long nxt = cjl + gridDim.x;
+  int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
+  bool have_n = nxt < p.total;
+  if (have_n) { item_geom(nxt, jn, jqn, Ln, tok0n); have_n = Ln > 0; }
+  float g_n = 0.f, b_n = 0.f;
+  if (have_n) {
+    if (tid == 0) issue_tiles(jn, jqn, tok0n);
+    if (!KDA && tid < Ln && tid < 64) {
+      g_n = p.g[(size_t)(tok0n + tid) * p.HV + jn];
+      b_n = p.beta[(size_t)(tok0n + tid) * p.HV + jn];
+    }
+  }
   {
-    // Q~^T is complete in the accumulator; the V tile is dead and receives its image.
+    // Q~^T and O_loc^T are complete in the accumulators; their images go where W^T and U^T were.
     float v[32];
     ld32(my_tmem, v);
-    store_half_row(v, rowq, hf, sm + OFF_V);
-    // O_loc image: rows 0..63 go to the K tile of feature half 0, rows 64..127 to that of half 1 (both dead)
+    store_half_row(v, rowq, hf, sm + OFF_WT);
     ld32(my_tmem + 64, v);
-    store_half_row(v, rowq & 63, hf, sm + OFF_KQ + (rowq >> 6) * 16384);
+    store_half_row(v, rowq, hf, sm + OFF_UT);
   }
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
   if (tid == 0) {
-    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_V, kImgBytes);
-    bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_KQ, 8192);
-    bulk_store(p.ws.ol + (size_t)cj * kImgBytes + 8192, sm + OFF_KQ + 16384, 8192);
+    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_WT, kImgBytes);
+    bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
     if constexpr (KDA) bulk_store(p.ws.kd + (size_t)cj * kImgBytes, sm + OFF_KD, kImgBytes);
     bulk_commit();
-    prev_cj = cjl;
   }
+  prev_cj = cjl;
   lph ^= 1;
+  cjl = nxt; have = have_n; j = jn; jq = jqn; L = Ln; tok0 = tok0n; g_pre = g_n; b_pre = b_n;
   HA_PROF(prep, 13);
   }  // work items
 

@@ -156,3 +156,20 @@ def test_tc_every_slice_width(nv, monkeypatch):
     a = ha.make_args(variant="gdn", dtype="bf16", batch=1, seqlen=inp["T"], hk=2, hv=4, dk=128, dv=128, num_seqs=3)
     assert ha.ha_la_prefill_path(a) == "tc"
     helpers.check_parity(inp)
+
+
+def test_concurrent_prep_and_chain_mode(monkeypatch):
+    """Opt-in mode: the chain kernel runs next to the persistent prep kernel and takes each chunk as soon
+    as its flag is published.  Same results as the sequential mode, bit for bit."""
+    w = synth.shrink(W["gdn_layer_4k"], seq_lens=[2048], hk=4, hv=4)
+    inp = synth.make_inputs(w, seed=37)
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", "0")
+    o_seq, h_seq, st_seq = helpers.run_gpu(inp)
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", "1")
+    o_con, h_con, st_con = helpers.run_gpu(inp)
+    o_con2, h_con2, _ = helpers.run_gpu(inp)
+    assert st_seq == 0 and st_con == 0
+    np.testing.assert_array_equal(o_con, o_seq)
+    np.testing.assert_array_equal(h_con, h_seq)
+    np.testing.assert_array_equal(o_con2, o_seq)
+    helpers.check_parity(inp)
