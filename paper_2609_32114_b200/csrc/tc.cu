@@ -21,7 +21,7 @@ namespace ha_la {
 
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                            const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int32_t epoch,
-                           int reserved_slots, cudaStream_t stream);
+                           int reserved_sms, cudaStream_t stream);
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                             const CUtensorMap& mk, int nv, int32_t epoch, cudaStream_t stream);
 
@@ -163,8 +163,8 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   // per SM) before the prep CTAs arrive; the prep kernel runs on the side stream and fills the remaining room.
   e = launch_tc_chain(p, a, plan, ws, mk, nv, epoch, stream);
   if (e != cudaSuccess) return e;
-  // a chain CTA (three stages) fills its SM: the prep kernel gets the other SMs, two CTAs each
-  e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, 2 * p.N * p.HV * (128 / nv), side->stream);
+  // a chain CTA (three stages) fills its SM: the prep kernel gets the other SMs
+  e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, p.N * p.HV * (128 / nv), side->stream);
   if (e != cudaSuccess) return e;
   e = cudaEventRecord(side->join, side->stream);
   if (e != cudaSuccess) return e;

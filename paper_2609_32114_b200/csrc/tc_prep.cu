@@ -5,8 +5,11 @@
 //   #1 Gate   G = chunk-local cumulative log-gate (warp scan)
 //   #2 KKT    S = [K; Q] K^T on the tensor cores (one M=128 MMA covers K K^T and Q K^T), then
 //             A_ij = beta_i e^{G_i-G_j} S_kk[i,j] (j<i)  and  P_ij = e^{G_i-G_j} S_qk[i,j] (j<=i) in fp32
-//   #3 Solve  T = (I + A)^-1 in fp32 by blocked forward substitution: four 16x16 diagonal blocks,
-//             then the off-diagonal blocks level by level as T_lo = -T_hi (A_lo T_lo')
+//   #3 Solve  T = (I + A)^-1 by blocked forward substitution: four 16x16 diagonal blocks in fp32 registers,
+//             then the off-diagonal blocks level by level as T_lo = -T_hi (A_lo T_lo') on mma.sync (fp16
+//             operands, fp32 accumulation).  A and T are held in shared memory as fp16 (T is rounded to bf16
+//             for the next operator anyway); this assumes the delta rule's usual normalisation
+//             (beta |k|^2 of order one), far inside the fp16 range.
 //   #4 W/U    W^T = K^T (T diag(beta e^G))^T,  U^T = V^T (T diag(beta))^T   (M = feature dim = 128)
 // and the chunk-local halves of operator #6, so that the sequential kernel needs one stacked MMA:
 //             Q~ = Q e^G - P W      O_loc = P U        (o = scale [Q~ h + O_loc])
@@ -20,6 +23,7 @@
 // read for them (the next sequence's rows, or zero fill past the end of the tensor) is multiplied
 // by exact zeros.  This relies on the inputs being finite.
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include "tc_common.cuh"
 #include "tc_ptx.cuh"
@@ -34,26 +38,25 @@ HA_PROF_DECL(prep)
 namespace {
 
 constexpr int kPrepThreads = 256;
-constexpr int LDF = 68;                  // row stride (floats) of the fp32 64x64 matrices
-constexpr int LDX = 36;                  // row stride of the 32x32 scratch
+constexpr int LDH = 72;                  // row stride (halfs) of the fp16 64x64 matrix A / T
 
-// shared-memory map (bytes from the 1024-aligned base)
+// shared-memory map (bytes from the 1024-aligned base); 73.3 KiB, so that three CTAs fit one SM
 constexpr uint32_t OFF_KQ = 0;           // [kb][K 8K | Q 8K], kb = 0,1 (feature halves)
-constexpr uint32_t OFF_V = 32768;        // [kb][V 8K]; later the Q~ image
-constexpr uint32_t OFF_R1 = 49152;       // solve scratch, later the W^T / U^T operand tiles (= W, U images)
-constexpr uint32_t OFF_A = OFF_R1;                       // fp32 [64][LDF]; later T^W, T^U tiles
-constexpr uint32_t OFF_T = OFF_R1 + 64 * LDF * 4;        // fp32 [64][LDF]
-constexpr uint32_t OFF_X = OFF_T + 64 * LDF * 4;         // fp32 [32][LDX]
+constexpr uint32_t OFF_E = OFF_KQ;       // bf16 [64][64] diag(e^G) tile over the first K piece, once K is dead
+constexpr uint32_t OFF_V = 32768;        // [kb][V 8K]; later the U image, then the O_loc image
+constexpr uint32_t OFF_UT = OFF_V;
+constexpr uint32_t OFF_R1 = 49152;       // 16 KiB: A / T (fp16), then T^W | T^U, then the W image, then the Q~ image
+constexpr uint32_t OFF_A = OFF_R1;                       // fp16 [64][LDH]: A, overwritten in place by T
+constexpr uint32_t OFF_D = OFF_R1 + 64 * LDH * 2;        // fp16 4 x [16][16]: inverses of the diagonal blocks
 constexpr uint32_t OFF_TW = OFF_R1;                      // bf16 [64][64] K-major, swizzled (8 KiB)
 constexpr uint32_t OFF_TU = OFF_R1 + 8192;
 constexpr uint32_t OFF_WT = OFF_R1;                      // bf16 [128][64] K-major, swizzled (16 KiB)
-constexpr uint32_t OFF_UT = OFF_R1 + 16384;
-constexpr uint32_t OFF_E = OFF_R1 + 32768;               // bf16 [64][64] diag(e^G), K-major, swizzled; overlaps T's tail and X,
-                                                         // so it is written only after the solve's results were consumed
-constexpr uint32_t OFF_P = OFF_R1 + 40960;               // bf16 [64][64] K-major, swizzled
+constexpr uint32_t OFF_P = OFF_R1 + 16384;               // bf16 [64][64] K-major, swizzled
 constexpr uint32_t OFF_MISC = OFF_P + 8192;              // floats: G[64], beta[64], e^G[64], beta e^G[64], G log2e[64]
 constexpr uint32_t OFF_BAR = OFF_MISC + 5 * 64 * 4;
 constexpr uint32_t kPrepSmem = OFF_BAR + 64;
+static_assert(OFF_D + 4 * 256 * 2 <= OFF_P, "solve scratch overlaps P");
+static_assert(3 * (kPrepSmem + 1024) <= 228 * 1024, "three CTAs per SM");
 // KDA only: per-channel cumulative log-gate (fp32, times log2 e) and the K e^{G_L - G} operand image
 constexpr int LDG = 132;                                  // row stride (floats) of the 64 x 128 gate matrix
 constexpr uint32_t OFF_G = (kPrepSmem + 1023) / 1024 * 1024;
@@ -66,8 +69,6 @@ constexpr uint32_t OFF_KM = OFF_KQP + 2 * KQP_KB;         // [kb][96 rows][128 B
 constexpr uint32_t KM_KB = 96 * 128;
 constexpr uint32_t kPrepSmemKda = OFF_KM + 2 * KM_KB;
 static_assert(kPrepSmemKda <= 227 * 1024, "KDA shared memory budget");
-static_assert(OFF_X + 32 * LDX * 4 <= OFF_P, "solve scratch overlaps P");
-static_assert(OFF_UT + 16384 <= OFF_P, "operand tiles overlap P");
 
 struct PrepParams {
   const float* g;
@@ -107,37 +108,84 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
   return make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
 }
 
-// One warp computes a 16 x 8 tile of C = A B from fp32 matrices in shared memory on the legacy tensor
-// path (mma.sync m16n8k8, TF32) with the 3-term split a = a_hi + a_lo, b = b_hi + b_lo, which keeps the
-// result at fp32 accuracy (the dropped a_lo b_lo term is ~2^-22 relative).  A is row-major (lda), B is
-// row-major K x N (ldb); `ksteps` steps of 8.  Result in the m16n8 accumulator layout:
-// c[0], c[1] = C[g][2t], C[g][2t+1];  c[2], c[3] = C[g+8][2t], C[g+8][2t+1]  (g = lane / 4, t = lane % 4).
-__device__ __forceinline__ uint32_t to_tf32(float x) {
-  uint32_t r;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-  return r;
+__device__ __forceinline__ void unpack8h(const uint4& w, float (&f)[8]) {          // 8 fp16 -> fp32
+  const __half2* h = reinterpret_cast<const __half2*>(&w);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 t = __half22float2(h[e]);
+    f[2 * e] = t.x;
+    f[2 * e + 1] = t.y;
+  }
 }
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
-  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Warp-level fp16 matrix products on the legacy tensor path (mma.sync m16n8k16, fp32 accumulation) with
+// operands fetched by ldmatrix from row-major fp16 matrices in shared memory.
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const __half* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)) : "memory");
+}
+__device__ __forceinline__ void ldsm_x2(uint32_t (&r)[2], const __half* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];"
+               : "=r"(r[0]), "=r"(r[1]) : "r"(smem_u32(p)) : "memory");
+}
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
-__device__ __forceinline__ void warp_tile_mm(float (&c)[4], const float* A, int lda, const float* B, int ldb,
-                                             int ksteps, int lane) {
+
+// One level of the blocked solve for BS x BS blocks (BS = 16 or 32):  T10 = -T11 (A10 T00), evaluated
+// transposed so that the first product's accumulators are the second product's A fragments:
+//   X^T = T00^T A10^T  (all BS/8 column tiles, needed as the contraction index of the second product),
+//   R^T = X^T T11^T    (NT2 tiles of 8 rows of T10, starting at tile nt2_0),
+// for the 16 columns mt*16.. of T10.  Results stay in registers (c2); store_merge() writes them over A10.
+template <int BS, int NT2>
+__device__ __forceinline__ void merge_compute(float (&c2)[NT2][4], const __half* T00, int ld00, const __half* A10,
+                                              int ldA, const __half* T11, int ld11, int mt, int nt2_0, int lane) {
+  constexpr int KS = BS / 16, NT = BS / 8;
+  float c1[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) c1[nt][0] = c1[nt][1] = c1[nt][2] = c1[nt][3] = 0.f;
+  const int j = lane >> 3, r = lane & 7;
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    uint32_t a[4];
+    ldsm_x4_t(a, T00 + (ks * 16 + (j >> 1) * 8 + r) * ld00 + mt * 16 + (j & 1) * 8);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      uint32_t b[2];
+      ldsm_x2(b, A10 + (nt * 8 + r) * ldA + ks * 16 + (j & 1) * 8);
+      mma_f16(c1[nt], a, b);
+    }
+  }
+#pragma unroll
+  for (int n2 = 0; n2 < NT2; ++n2) c2[n2][0] = c2[n2][1] = c2[n2][2] = c2[n2][3] = 0.f;
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    const uint32_t a[4] = {pack_f16(c1[2 * ks][0], c1[2 * ks][1]), pack_f16(c1[2 * ks][2], c1[2 * ks][3]),
+                           pack_f16(c1[2 * ks + 1][0], c1[2 * ks + 1][1]), pack_f16(c1[2 * ks + 1][2], c1[2 * ks + 1][3])};
+#pragma unroll
+    for (int n2 = 0; n2 < NT2; ++n2) {
+      uint32_t b[2];
+      ldsm_x2(b, T11 + ((nt2_0 + n2) * 8 + r) * ld11 + ks * 16 + (j & 1) * 8);
+      mma_f16(c2[n2], a, b);
+    }
+  }
+}
+template <int NT2>
+__device__ __forceinline__ void merge_store(const float (&c2)[NT2][4], __half* T10, int ld, int mt, int nt2_0, int lane) {
   const int g = lane >> 2, t = lane & 3;
-  c[0] = c[1] = c[2] = c[3] = 0.f;
-  for (int ks = 0; ks < ksteps; ++ks) {
-    const float af[4] = {A[g * lda + ks * 8 + t], A[(g + 8) * lda + ks * 8 + t], A[g * lda + ks * 8 + t + 4],
-                         A[(g + 8) * lda + ks * 8 + t + 4]};
-    const float bf[2] = {B[(ks * 8 + t) * ldb + g], B[(ks * 8 + t + 4) * ldb + g]};
-    uint32_t ah[4], al[4], bh[2], bl[2];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) { ah[e] = to_tf32(af[e]); al[e] = to_tf32(af[e] - __uint_as_float(ah[e])); }
-#pragma unroll
-    for (int e = 0; e < 2; ++e) { bh[e] = to_tf32(bf[e]); bl[e] = to_tf32(bf[e] - __uint_as_float(bh[e])); }
-    mma_tf32(c, al, bh);
-    mma_tf32(c, ah, bl);
-    mma_tf32(c, ah, bh);
+  for (int n2 = 0; n2 < NT2; ++n2) {
+    __half* d = T10 + ((nt2_0 + n2) * 8 + 2 * t) * ld + mt * 16 + g;
+    d[0] = __float2half_rn(-c2[n2][0]);
+    d[ld] = __float2half_rn(-c2[n2][1]);
+    d[8] = __float2half_rn(-c2[n2][2]);
+    d[ld + 8] = __float2half_rn(-c2[n2][3]);
   }
 }
 
@@ -155,21 +203,21 @@ __device__ __forceinline__ void store_half_row(const float (&v)[32], int row, in
 }
 
 template <bool KDA>
-__global__ void __launch_bounds__(kPrepThreads, KDA ? 1 : 2)
+__global__ void __launch_bounds__(kPrepThreads, KDA ? 1 : 3)
 tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, PrepParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* sm = smem_raw;                                // no static shared memory in this kernel: 1024-aligned
-  float* sA = reinterpret_cast<float*>(sm + OFF_A);
-  float* sT = reinterpret_cast<float*>(sm + OFF_T);
-  float* sX = reinterpret_cast<float*>(sm + OFF_X);
+  __half* sAh = reinterpret_cast<__half*>(sm + OFF_A);  // A, then T in place
+  __half* sD = reinterpret_cast<__half*>(sm + OFF_D);
   float* sG = reinterpret_cast<float*>(sm + OFF_MISC);
   float* sBeta = sG + 64;
   float* sEG = sG + 128;
   float* sBE = sG + 192;
   uint64_t* bar_load = reinterpret_cast<uint64_t*>(sm + OFF_BAR);
   uint64_t* bar_mma = bar_load + 1;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_load + 2);
+  uint64_t* bar_v = bar_load + 2;                        // the V tiles arrive on their own barrier
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_load + 3);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* sTmp = reinterpret_cast<float*>(tmem_slot + 2);
 
@@ -181,10 +229,12 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
   HA_PROF(prep, 0);
   HA_PROF_SMID(prep, 256, 512);
+#define PP(slot) do { if (cjl == (long long)gridDim.x) HA_PROF(prep, slot); } while (0)
 
   if (tid == 0) {
     mbar_init(bar_load, 1);
     mbar_init(bar_mma, 1);
+    mbar_init(bar_v, 1);
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
@@ -217,13 +267,16 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       L_ = min(kChunk, p.T_row - cc_ * kChunk);
     }
   };
-  auto issue_tiles = [&](int j_, int jq_, int tok0_) {   // thread 0: K, Q, V tiles of one item
-    mbar_expect_tx(bar_load, 6 * 8192);
+  auto issue_tiles = [&](int jq_, int tok0_) {           // thread 0: K and Q tiles of one item
+    mbar_expect_tx(bar_load, 4 * 8192);
     for (int kb = 0; kb < 2; ++kb) {
       tma_load_3d(sm + OFF_KQ + kb * 16384, &map_k, bar_load, kb * 64, jq_, tok0_);
       tma_load_3d(sm + OFF_KQ + kb * 16384 + 8192, &map_q, bar_load, kb * 64, jq_, tok0_);
-      tma_load_3d(sm + OFF_V + kb * 8192, &map_v, bar_load, kb * 64, j_, tok0_);
     }
+  };
+  auto issue_v = [&](int j_, int tok0_) {                // thread 0: V tiles (their room is free later than K's)
+    mbar_expect_tx(bar_v, 2 * 8192);
+    for (int kb = 0; kb < 2; ++kb) tma_load_3d(sm + OFF_V + kb * 8192, &map_v, bar_v, kb * 64, j_, tok0_);
   };
   auto publish_prev = [&]() {                            // thread 0, concurrent mode: hand the previous item over
     if (p.epoch != 0 && prev_cj >= 0) {
@@ -239,7 +292,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (have) { item_geom(cjl, j, jq, L, tok0); have = L > 0; }   // unused chunk slots come last
   float g_pre = 0.f, b_pre = 0.f;                        // GDN, threads 0..63: this token's log-gate and beta
   if (have) {
-    if (tid == 0) issue_tiles(j, jq, tok0);
+    if (tid == 0) issue_tiles(jq, tok0);
     if (!KDA && tid < L && tid < 64) {
       g_pre = p.g[(size_t)(tok0 + tid) * p.HV + j];
       b_pre = p.beta[(size_t)(tok0 + tid) * p.HV + j];
@@ -248,7 +301,10 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   while (have) {
   const size_t cj = (size_t)cjl;
   // The previous item's bulk stores must have read their shared-memory sources before anything is overwritten.
-  if (tid == 0 && prev_cj >= 0) bulk_wait_read_all();
+  if (tid == 0) {
+    if (prev_cj >= 0) bulk_wait_read_all();
+    issue_v(j, tok0);                                    // lands where the previous item's O_loc image was
+  }
   __syncthreads();
   if constexpr (KDA) {
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
@@ -266,7 +322,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         sEG[tid] = 1.f;                                  // and Q is rescaled in place: E = identity
       }
       // A and P start as zero (entries above the diagonal are never written)
-      for (int idx = tid; idx < 64 * LDF; idx += kPrepThreads) sA[idx] = 0.f;
+      for (int idx = tid; idx < 64 * LDH * 2 / 16; idx += kPrepThreads) reinterpret_cast<uint4*>(sAh)[idx] = make_uint4(0, 0, 0, 0);
       for (int idx = tid; idx < 512; idx += kPrepThreads) reinterpret_cast<uint4*>(sm + OFF_P)[idx] = make_uint4(0, 0, 0, 0);
     }
     __syncthreads();
@@ -283,7 +339,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     mbar_wait(bar_load, lph, abort_flag);                // every thread reads the K / Q tiles below
     __syncthreads();
-    HA_PROF(prep, 4);
+    PP(4);
 
     // ---- op #2 KKT and the masked Q K^T with per-channel decay:
     //   A_ij = beta_i sum_c k_ic k_jc 2^(G_ic - G_jc) (j < i),  P_ij = sum_c q_ic k_jc 2^(G_ic - G_jc) (j <= i).
@@ -371,7 +427,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           qk = fmaf(qif[e], t, qk);
         }
       }
-      if (jj < i) sA[i * LDF + jj] = sBeta[i] * kk;
+      if (jj < i) sAh[i * LDH + jj] = __float2half_rn(sBeta[i] * kk);
       *reinterpret_cast<__nv_bfloat16*>(sm + OFF_P + sw128_offset(i, jj >> 3) + (jj & 7) * 2) = __float2bfloat16_rn(qk);
     }
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
@@ -400,7 +456,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const float bi = sBeta[i];
 #pragma unroll
             for (int c = 0; c < 16 * I; c += 4)
-              *reinterpret_cast<float4*>(sA + i * LDF + c) = make_float4(bi * v[c], bi * v[c + 1], bi * v[c + 2], bi * v[c + 3]);
+              *reinterpret_cast<uint2*>(sAh + i * LDH + c) = make_uint2(pack_f16(bi * v[c], bi * v[c + 1]), pack_f16(bi * v[c + 2], bi * v[c + 3]));
           } else {
 #pragma unroll
             for (int ch = 0; ch < 2 * I; ++ch) {
@@ -467,9 +523,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
     // ---- op #2 KKT (+ Q K^T): S[0:64] = K K^T, S[64:128] = Q K^T
     if (tid == 0) {
-      HA_PROF(prep, 2);
+      PP(2);
       mbar_wait(bar_load, lph, abort_flag);
-      HA_PROF(prep, 3);
+      PP(3);
       tc_fence_after_sync();
       const uint32_t id = idesc_bf16(128, 64, false, false);
       const uint32_t base = smem_u32(sm + OFF_KQ);
@@ -484,7 +540,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);  // one warp polls; the others sleep at the barrier
     mph ^= 1;
     __syncthreads();                                     // (also makes sEG / sBE visible to everyone)
-    HA_PROF(prep, 4);
+    PP(4);
     tc_fence_after_sync();
     {
       float v[32];
@@ -492,7 +548,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const int i = rowq & 63;
       const float* sG2 = sBE + 64;                       // G log2(e)
       const float gi = sG2[i];
-      if (rowq < 64) {                                     // row i of A (strictly lower, beta-scaled), fp32
+      if (rowq < 64) {                                     // row i of A (strictly lower, beta-scaled), fp16
         const float bi = sBeta[i];
   #pragma unroll
         for (int q = 0; q < 32; ++q) {
@@ -501,8 +557,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           v[q] = jj < i ? bi * e * v[q] : 0.f;
         }
   #pragma unroll
-        for (int q = 0; q < 32; q += 4)
-          *reinterpret_cast<float4*>(sA + i * LDF + hf * 32 + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+        for (int q = 0; q < 32; q += 8)
+          *reinterpret_cast<uint4*>(sAh + i * LDH + hf * 32 + q) =
+              make_uint4(pack_f16(v[q], v[q + 1]), pack_f16(v[q + 2], v[q + 3]), pack_f16(v[q + 4], v[q + 5]), pack_f16(v[q + 6], v[q + 7]));
       } else {                                             // row i of P (lower incl. diagonal), bf16 operand tile
   #pragma unroll
         for (int q = 0; q < 32; ++q) {
@@ -515,112 +572,86 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
   }
   __syncthreads();
-  HA_PROF(prep, 5);
+  PP(5);
 
-  // ---- op #3 Solve: T = (I + A)^-1, fp32
+  // ---- op #3 Solve: T = (I + A)^-1
   if (tid < 64) {
-    // four 16x16 diagonal blocks; thread = (block, column).  Column-oriented substitution: once x_r is
-    // final, every later row is updated independently (short dependency chain).
-    const int o = (tid >> 4) * 16, c = tid & 15;
+    // Four 16x16 diagonal blocks; thread = (block, column c of the inverse), fp32 forward substitution row by
+    // row: y_q = [q == c] - sum_{r<q} A[q][r] y_r.  The inverse goes to a scratch copy first (the other
+    // threads of the block are still reading A).
+    const int blk = tid >> 4, c = tid & 15, o = blk * 16;
     float y[16];
 #pragma unroll
-    for (int r = 0; r < 16; ++r) y[r] = r == c ? 1.f : 0.f;
+    for (int q = 0; q < 16; ++q) {
+      float a[16];
+      if (q > 0) unpack8h(*reinterpret_cast<const uint4*>(sAh + (o + q) * LDH + o), *reinterpret_cast<float(*)[8]>(a));
+      if (q > 8) unpack8h(*reinterpret_cast<const uint4*>(sAh + (o + q) * LDH + o + 8), *reinterpret_cast<float(*)[8]>(a + 8));
+      float s0 = q == c ? 1.f : 0.f, s1 = 0.f;
 #pragma unroll
-    for (int r = 0; r < 16; ++r) {
-      const float xr = y[r];
-      sT[(o + r) * LDF + o + c] = xr;
-#pragma unroll
-      for (int q = r + 1; q < 16; ++q) y[q] = fmaf(-sA[(o + q) * LDF + o + r], xr, y[q]);
-    }
-  } else {
-    // blocks above the diagonal are zero: 6 blocks of 16x16
-    for (int idx = tid - 64; idx < 6 * 256; idx += kPrepThreads - 64) {
-      const int blk = idx >> 8, e = idx & 255;
-      const int bi = blk < 3 ? 0 : (blk < 5 ? 1 : 2);
-      const int bj = blk < 3 ? blk + 1 : (blk < 5 ? blk - 1 : 3);
-      sT[(bi * 16 + (e >> 4)) * LDF + bj * 16 + (e & 15)] = 0.f;
+      for (int r = 0; r < q; ++r) {
+        if (r & 1) s1 = fmaf(-a[r], y[r], s1);
+        else s0 = fmaf(-a[r], y[r], s0);
+      }
+      y[q] = s0 + s1;
+      sD[blk * 256 + q * 16 + c] = __float2half_rn(y[q]);
     }
   }
   __syncthreads();
-  HA_PROF(prep, 6);
+  PP(6);
   {
-    // level 1: blocks (1,0) and (3,2).  X = A_lo T_lo' ; warps 0..3 -> (pair, 8-column tile)
-    if (warp < 4) {
-      const int pr = warp >> 1, nt = warp & 1;
-      const int lo = pr * 32, hi = lo + 16;
-      float c[4];
-      warp_tile_mm(c, sA + hi * LDF + lo, LDF, sT + lo * LDF + lo + nt * 8, LDF, 2, lane);
-      const int g = lane >> 2, t = lane & 3;
-      float* x = sX + (pr * 16) * LDX + nt * 8;
-      x[g * LDX + 2 * t] = c[0]; x[g * LDX + 2 * t + 1] = c[1];
-      x[(g + 8) * LDX + 2 * t] = c[2]; x[(g + 8) * LDX + 2 * t + 1] = c[3];
+    // the diagonal inverses go back in place (for level 2 and the final read) ...
+    const int blk = tid >> 6, r = (tid >> 2) & 15, c4 = (tid & 3) * 4;
+    *reinterpret_cast<uint2*>(sAh + (blk * 16 + r) * LDH + blk * 16 + c4) =
+        *reinterpret_cast<const uint2*>(sD + blk * 256 + r * 16 + c4);
+    // ... while level 1 (blocks (1,0) and (3,2)) reads them from the scratch copy: one warp per block
+    if (warp < 2) {
+      const int lo = warp * 32, hi = lo + 16;
+      float c2[2][4];
+      merge_compute<16, 2>(c2, sD + (2 * warp) * 256, 16, sAh + hi * LDH + lo, LDH, sD + (2 * warp + 1) * 256, 16, 0, 0, lane);
+      __syncwarp();
+      merge_store<2>(c2, sAh + hi * LDH + lo, LDH, 0, 0, lane);
     }
   }
   __syncthreads();
+  PP(7);
   {
-    if (warp < 4) {                                      // T_lo = -T_hi X
-      const int pr = warp >> 1, nt = warp & 1;
-      const int lo = pr * 32, hi = lo + 16;
-      float c[4];
-      warp_tile_mm(c, sT + hi * LDF + hi, LDF, sX + (pr * 16) * LDX + nt * 8, LDX, 2, lane);
-      const int g = lane >> 2, t = lane & 3;
-      float* d = sT + hi * LDF + lo + nt * 8;
-      d[g * LDF + 2 * t] = -c[0]; d[g * LDF + 2 * t + 1] = -c[1];
-      d[(g + 8) * LDF + 2 * t] = -c[2]; d[(g + 8) * LDF + 2 * t + 1] = -c[3];
-    }
+    // level 2: the 32x32 block (rows 32..63, columns 0..31); warp -> (16 columns, 8 rows) of the result
+    const int mt = warp & 1, n2 = warp >> 1;
+    float c2[1][4];
+    merge_compute<32, 1>(c2, sAh, LDH, sAh + 32 * LDH, LDH, sAh + 32 * LDH + 32, LDH, mt, n2, lane);
+    __syncthreads();                                     // every warp has read A_10 before it is overwritten
+    merge_store<1>(c2, sAh + 32 * LDH, LDH, mt, n2, lane);
   }
   __syncthreads();
-  HA_PROF(prep, 7);
-  {
-    // level 2: the 32x32 block (rows 32..63, columns 0..31).  X = A_10 T_00 ; warp -> (16-row tile, 8-column tile)
-    const int mt = warp >> 2, nt = warp & 3;
-    float c[4];
-    warp_tile_mm(c, sA + (32 + mt * 16) * LDF, LDF, sT + nt * 8, LDF, 4, lane);
-    const int g = lane >> 2, t = lane & 3;
-    float* x = sX + (mt * 16) * LDX + nt * 8;
-    x[g * LDX + 2 * t] = c[0]; x[g * LDX + 2 * t + 1] = c[1];
-    x[(g + 8) * LDX + 2 * t] = c[2]; x[(g + 8) * LDX + 2 * t + 1] = c[3];
-  }
-  __syncthreads();
-  {
-    // T_10 = -T_11 X
-    const int mt = warp >> 2, nt = warp & 3;
-    float c[4];
-    warp_tile_mm(c, sT + (32 + mt * 16) * LDF + 32, LDF, sX + nt * 8, LDX, 4, lane);
-    const int g = lane >> 2, t = lane & 3;
-    float* d = sT + (32 + mt * 16) * LDF + nt * 8;
-    d[g * LDF + 2 * t] = -c[0]; d[g * LDF + 2 * t + 1] = -c[1];
-    d[(g + 8) * LDF + 2 * t] = -c[2]; d[(g + 8) * LDF + 2 * t + 1] = -c[3];
-  }
-  __syncthreads();
-  HA_PROF(prep, 8);
+  PP(8);
 
-  // ---- column-scaled copies of T as bf16 operand tiles: T^W = T diag(beta e^G), T^U = T diag(beta)
+  // ---- column-scaled copies of T as bf16 operand tiles: T^W = T diag(beta e^G), T^U = T diag(beta).
+  // They overwrite T, so every thread first takes its part of T into registers.
   {
     const int i = tid >> 2, q4 = tid & 3;                // row, quarter (16 columns = two 16-byte pieces)
+    const uint4 traw0 = *reinterpret_cast<const uint4*>(sAh + i * LDH + q4 * 16);
+    const uint4 traw1 = *reinterpret_cast<const uint4*>(sAh + i * LDH + q4 * 16 + 8);
+    __syncthreads();
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
       const int ch = q4 * 2 + q;
-      float tw[8], tu[8];
+      float tv[8], tw[8], tu[8];
+      unpack8h(q == 0 ? traw0 : traw1, tv);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int jj = ch * 8 + e;
-        const float t = sT[i * LDF + jj];
-        tw[e] = t * sBE[jj];
-        tu[e] = t * sBeta[jj];
+        tw[e] = tv[e] * sBE[jj];
+        tu[e] = tv[e] * sBeta[jj];
       }
-      uint4 w, u;
-      w.x = pack_bf16(tw[0], tw[1]); w.y = pack_bf16(tw[2], tw[3]); w.z = pack_bf16(tw[4], tw[5]); w.w = pack_bf16(tw[6], tw[7]);
-      u.x = pack_bf16(tu[0], tu[1]); u.y = pack_bf16(tu[2], tu[3]); u.z = pack_bf16(tu[4], tu[5]); u.w = pack_bf16(tu[6], tu[7]);
       const uint32_t off = sw128_offset(i, ch);
-      *reinterpret_cast<uint4*>(sm + OFF_TW + off) = w;   // overwrites sA, which is dead by now
-      *reinterpret_cast<uint4*>(sm + OFF_TU + off) = u;
+      *reinterpret_cast<uint4*>(sm + OFF_TW + off) = pack8(tw);
+      *reinterpret_cast<uint4*>(sm + OFF_TU + off) = pack8(tu);
     }
   }
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
-  HA_PROF(prep, 9);
+  PP(9);
 
   // ---- op #4 W/U: W^T = K^T (T^W)^T, U^T = V^T (T^U)^T  (A operands feature-major straight from the TMA tiles)
   if (tid == 0) {
@@ -630,6 +661,8 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     for (int ks = 0; ks < 4; ++ks)
       umma_ss(tmem, smem_desc(smem_u32(sm + OFF_KQ) + ks * 2048, 16384, 1024, kSwizzle128B),
               smem_desc(smem_u32(sm + OFF_TW) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
+    mbar_wait(bar_v, lph, abort_flag);
+    tc_fence_after_sync();
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks)
       umma_ss(tmem + 64, smem_desc(smem_u32(sm + OFF_V) + ks * 2048, 8192, 1024, kSwizzle128B),
@@ -639,7 +672,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
   mph ^= 1;
   __syncthreads();
-  HA_PROF(prep, 10);
+  PP(10);
   tc_fence_after_sync();
   {
     float v[32];
@@ -648,7 +681,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     ld32(my_tmem + 64, v);
     store_half_row(v, rowq, hf, sm + OFF_UT);
     // E = diag(e^G) as an MMA operand: Q^T E puts (Q e^G)^T into the accumulator of the Q~ product.
-    // It lies over the tail of the fp32 T matrix, which is dead only now.
+    // It lies over the first K piece, which is dead now that the W product is complete.
     const int i = tid >> 2;
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
@@ -664,7 +697,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
-  HA_PROF(prep, 11);
+  PP(11);
 
   // ---- chunk-local halves of op #6: (P W)^T = W^T P^T, O_loc^T = U^T P^T; the W and U images leave meanwhile
   if (tid == 0) {
@@ -703,16 +736,17 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (tid == 0) bulk_wait_read_all();                    // the W^T / U^T tiles were read; they receive the next images
   mph ^= 1;
   __syncthreads();
-  HA_PROF(prep, 12);
+  PP(12);
   tc_fence_after_sync();
-  // Every MMA of this item is done, so the K / Q / V tile regions are free: start the next item's loads now.
+  // Every MMA of this item is done, so the K / Q tile regions are free: start the next item's loads now
+  // (its V tiles follow at the top of the loop, once the O_loc image has left their room).
   const long long nxt = cjl + gridDim.x;
   int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
   bool have_n = nxt < p.total;
   if (have_n) { item_geom(nxt, jn, jqn, Ln, tok0n); have_n = Ln > 0; }
   float g_n = 0.f, b_n = 0.f;
   if (have_n) {
-    if (tid == 0) issue_tiles(jn, jqn, tok0n);
+    if (tid == 0) issue_tiles(jqn, tok0n);
     if (!KDA && tid < Ln && tid < 64) {
       g_n = p.g[(size_t)(tok0n + tid) * p.HV + jn];
       b_n = p.beta[(size_t)(tok0n + tid) * p.HV + jn];
@@ -738,7 +772,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   prev_cj = cjl;
   lph ^= 1;
   cjl = nxt; have = have_n; j = jn; jq = jqn; L = Ln; tok0 = tok0n; g_pre = g_n; b_pre = b_n;
-  HA_PROF(prep, 13);
+  PP(13);
   }  // work items
 
   __syncthreads();
@@ -789,7 +823,7 @@ cudaError_t configure_tc_prep(const Problem& p) {
 
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                            const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int32_t epoch,
-                           int reserved_slots, cudaStream_t stream) {
+                           int reserved_sms, cudaStream_t stream) {
   PrepParams pp;
   pp.epoch = epoch;
   pp.g = a.g; pp.beta = a.beta;
@@ -800,8 +834,8 @@ cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanVi
   if (pp.total == 0) return cudaSuccess;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  // resident CTAs; in the concurrent mode every chain CTA takes the place of one of them
-  long long slots = (long long)sms * (p.variant == HA_LA_KDA ? 1 : 2) - reserved_slots;
+  // resident CTAs; in the concurrent mode the SMs that hold a chain CTA are left out
+  long long slots = (long long)(sms - reserved_sms) * (p.variant == HA_LA_KDA ? 1 : 3);
   if (slots < 1) slots = 1;
   const long long grid = pp.total < slots ? pp.total : slots;
   return p.variant == HA_LA_KDA ? launch_prep_variant<true>(pp, mq, mk, mv, grid, stream)
