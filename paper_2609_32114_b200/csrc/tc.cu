@@ -26,7 +26,7 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
                             const CUtensorMap& mk, int nv, int32_t epoch, cudaStream_t stream);
 
 cudaError_t configure_tc_prep(const Problem& p);
-cudaError_t configure_tc_chain(const Problem& p, int nv, bool concurrent);
+cudaError_t configure_tc_chain(const Problem& p, int nv);
 
 namespace {
 
@@ -145,7 +145,7 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   // Configure (and load) both kernels before anything is enqueued.
   cudaError_t ce = configure_tc_prep(p);
   if (ce != cudaSuccess) return ce;
-  ce = configure_tc_chain(p, nv, false);
+  ce = configure_tc_chain(p, nv);
   if (ce != cudaSuccess) return ce;
   if (!side) {
     cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, 0, 0, stream);

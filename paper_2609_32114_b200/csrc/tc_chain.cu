@@ -14,9 +14,10 @@
 //   MMA2  D2[128 x NV] = K^T U~              (A = the raw K tile, feature-major, by TMA)
 //         all threads    : h <- e^{G_L} h + D2                   (op #5 update, in place)
 //
-// Warp roles: warps 0-3 compute (thread t <-> tensor-memory lane t), warp 4 produces (keeps the next
-// chunks' operands in flight through a ring of shared-memory stages: 1-D bulk copies + one TMA
-// tile), warp 5 issues the MMAs.  A tcgen05.mma costs the issuing thread about 65 cycles whatever
+// Warp roles: 4 CG compute warps (warp w <-> tensor-memory lanes 32 (w % 4).., column group w / 4 of the
+// slice: CG groups of NV / CG value channels, so that wide slices do not lengthen the epilogues), then one
+// producer warp (keeps the next chunks' operands in flight through a ring of shared-memory stages: 1-D
+// bulk copies + one TMA tile) and one warp that issues the MMAs.  A tcgen05.mma costs the issuing thread about 65 cycles whatever
 // its N <= 128, so issue runs on its own warp and is told "operand ready" with arrive-only named
 // barriers; the compute warps never wait for issue, only for completion (mbarriers).  Every
 // mbarrier wait is bounded.
@@ -34,7 +35,7 @@ HA_PROF_DECL(chain)
 
 namespace {
 
-constexpr int kChainThreads = 192;       // 4 compute warps + producer warp + MMA warp
+constexpr int chain_threads(int cg) { return (4 * cg + 2) * 32; }   // compute warps + producer warp + MMA warp
 
 template <int NV, int S_> struct ChainCfg {
   static constexpr int kStages = S_;
@@ -114,8 +115,8 @@ __device__ __forceinline__ void ld32f(uint32_t taddr, float (&v)[32]) {
 }
 
 // named barriers (0 is __syncthreads)
-constexpr int BAR_H_READY = 1;   // 128 compute threads arrive, MMA warp syncs: bf16 h is in shared memory
-constexpr int BAR_U_READY = 2;   // 64 U~ writers arrive, MMA warp syncs: U~ operand is in shared memory
+constexpr int BAR_H_READY = 1;   // all compute threads arrive, MMA warp syncs: bf16 h is in shared memory
+constexpr int BAR_U_READY = 2;   // the U~ writers (half of them) arrive, MMA warp syncs: U~ operand is in shared memory
 __device__ __forceinline__ void named_arrive(int id, int count) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
@@ -123,11 +124,15 @@ __device__ __forceinline__ void named_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
-template <int NV, bool KDA, int S>
-__global__ void __launch_bounds__(kChainThreads, 1)
+template <int NV, bool KDA, int S, int CG>
+__global__ void __launch_bounds__(chain_threads(CG), 1)
 tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   using Cfg = ChainCfg<NV, S>;
   constexpr int NSL = 128 / NV;
+  constexpr int NVT = NV / CG;                           // value channels per compute thread
+  constexpr int NCOMP = 128 * CG;                        // compute threads
+  constexpr int W_PROD = 4 * CG, W_MMA = 4 * CG + 1;
+  static_assert(NVT % 32 == 0, "column groups are multiples of 32 channels");
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* sm = smem_raw;                                // no static shared memory in this kernel: 1024-aligned
   uint64_t* bar_full = reinterpret_cast<uint64_t*>(sm + Cfg::OFF_BAR);     // [S]  producer -> everyone
@@ -150,7 +155,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
 
   HA_PROF_SMID(chain, 768, 128);
   if (tid == 0) {
-    for (int i = 0; i < S; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 128); }
+    for (int i = 0; i < S; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], NCOMP); }
     mbar_init(bar_mma1, 1);
     mbar_init(bar_mma2, 1);
     *abort_flag = 0;
@@ -166,7 +171,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   uint8_t* sH = sm + Cfg::OFF_H;
   uint8_t* sUt = sm + Cfg::OFF_UT;
 
-  if (warp == 4) {
+  if (warp == W_PROD) {
     // ------------------------------------------------------------ producer
     if ((tid & 31) == 0) {
       for (int c = 0; c < nchunks; ++c) {
@@ -196,7 +201,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
         }
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == W_MMA) {
     // ------------------------------------------------------------ MMA issue (lane 0 issues; the warp keeps the barriers)
     const uint32_t id = idesc_bf16(128, NV, true, true);
     const uint64_t dH = brow_desc0<NV, 128>(smem_u32(sH));
@@ -208,7 +213,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
       const uint64_t dWQ = smem_desc(stage + Cfg::OFF_WQ, 16384, 1024, kSwizzle128B);
       const uint64_t dK = smem_desc(stage + Cfg::OFF_K, 8192, 1024, kSwizzle128B);
       if (lead) mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
-      named_sync(BAR_H_READY, 128 + 32);                 // h (bf16) of the previous chunk is in sH
+      named_sync(BAR_H_READY, NCOMP + 32);               // h (bf16) of the previous chunk is in sH
       if (lead) {
         tc_fence_after_sync();
 #pragma unroll
@@ -216,7 +221,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
           umma_ss(TM1, dWQ + ks * (2048u >> 4), dH + ks * brow_step16<NV>(), id, ks > 0);
         umma_commit(bar_mma1);
       }
-      named_sync(BAR_U_READY, 64 + 32);                  // U~ is in sUt
+      named_sync(BAR_U_READY, NCOMP / 2 + 32);           // U~ is in sUt
       if (lead) {
         tc_fence_after_sync();
 #pragma unroll
@@ -226,30 +231,32 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
       }
     }
   } else {
-    // ------------------------------------------------------------ compute (threads 0..127)
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
-    float h[NV];                                         // state row `tid` (key channel), NV value channels
+    // ------------------------------------------------------------ compute
+    const int row = tid & 127;                           // tensor-memory lane = state row (key channel) / D1 row
+    const int cg0 = (warp >> 2) * NVT;                   // first value channel of this thread's column group
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    float h[NVT];                                        // state row `row`, NVT value channels
     {
-      const size_t base = (((size_t)n * p.HV + j) * 128 + tid) * 128 + (size_t)slice * NV;
+      const size_t base = (((size_t)n * p.HV + j) * 128 + row) * 128 + (size_t)slice * NV + cg0;
 #pragma unroll
-      for (int q = 0; q < NV; q += 4) {
+      for (int q = 0; q < NVT; q += 4) {
         float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
         if (p.h0) v4 = *reinterpret_cast<const float4*>(p.h0 + base + q);
         h[q] = v4.x; h[q + 1] = v4.y; h[q + 2] = v4.z; h[q + 3] = v4.w;
       }
     }
 #pragma unroll
-    for (int c0 = 0; c0 < NV; c0 += 32) {
+    for (int c0 = 0; c0 < NVT; c0 += 32) {
       float t[32];
 #pragma unroll
       for (int q = 0; q < 32; ++q) t[q] = h[c0 + q];
-      store_brow32<NV, 128>(sH, tid, c0, t);
+      store_brow32<NV, 128>(sH, row, cg0 + c0, t);
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
-    named_arrive(BAR_H_READY, 128 + 32);
+    named_arrive(BAR_H_READY, NCOMP + 32);
 
-    const int i = tid & 63;                              // token row handled in the first epilogue
+    const int i = row & 63;                              // token row handled in the first epilogue
     for (int c = 0; c < nchunks; ++c) {
       const int st = c % S;
       const uint8_t* stage = sm + st * Cfg::kStageB;
@@ -262,35 +269,35 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
       // operands of the first epilogue that do not depend on the MMA, fetched while it runs
       const float* sc = reinterpret_cast<const float*>(stage + Cfg::OFF_SC);
       const float dec = sc[i];
-      const float gam = sc[64 + tid];
+      const float gam = sc[64 + row];
       float pre[32];
-      load_img32(stage + (tid < 64 ? Cfg::OFF_U : Cfg::OFF_O), i, 0, pre);
+      load_img32(stage + (row < 64 ? Cfg::OFF_U : Cfg::OFF_O), i, cg0, pre);
 
       mbar_wait(bar_mma1, ph, abort_flag);
       HA_PROF(chain, 8 * c + 2);
       tc_fence_after_sync();
-      if (tid < 64) {                                    // U~ rows: (U - W h) e^{G_L - G_i}, the MMA2 operand
+      if (row < 64) {                                    // U~ rows: (U - W h) e^{G_L - G_i}, the MMA2 operand
 #pragma unroll
-        for (int c0 = 0; c0 < NV; c0 += 32) {
+        for (int c0 = 0; c0 < NVT; c0 += 32) {
           float d[32];
-          ld32f(TM1 + lane_base + c0, d);
-          if (c0 > 0) load_img32(stage + Cfg::OFF_U, i, c0, pre);
+          ld32f(TM1 + lane_base + cg0 + c0, d);
+          if (c0 > 0) load_img32(stage + Cfg::OFF_U, i, cg0 + c0, pre);
 #pragma unroll
           for (int q = 0; q < 32; ++q) d[q] = (pre[q] - d[q]) * dec;
-          store_brow32<NV, 64>(sUt, i, c0, d);
+          store_brow32<NV, 64>(sUt, i, cg0 + c0, d);
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
-        named_arrive(BAR_U_READY, 64 + 32);
+        named_arrive(BAR_U_READY, NCOMP / 2 + 32);
         HA_PROF(chain, 8 * c + 3);
       } else {                                           // output rows: o = scale (O_loc + Q~ h)  (op #6)
         __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
-                              ((size_t)(tok0 + c * kChunk + i) * p.HV + j) * 128 + (size_t)slice * NV;
+                              ((size_t)(tok0 + c * kChunk + i) * p.HV + j) * 128 + (size_t)slice * NV + cg0;
 #pragma unroll
-        for (int c0 = 0; c0 < NV; c0 += 32) {
+        for (int c0 = 0; c0 < NVT; c0 += 32) {
           float d[32];
-          ld32f(TM1 + lane_base + c0, d);
-          if (c0 > 0) load_img32(stage + Cfg::OFF_O, i, c0, pre);
+          ld32f(TM1 + lane_base + cg0 + c0, d);
+          if (c0 > 0) load_img32(stage + Cfg::OFF_O, i, cg0 + c0, pre);
 #pragma unroll
           for (int q = 0; q < 32; ++q) d[q] = p.scale * (pre[q] + d[q]);
           if (i < L) {
@@ -310,40 +317,40 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
       tc_fence_after_sync();
       mbar_arrive(&bar_empty[st]);                       // this thread and both MMAs are done with the stage
 #pragma unroll
-      for (int c0 = 0; c0 < NV; c0 += 32) {
+      for (int c0 = 0; c0 < NVT; c0 += 32) {
         float d[32];
-        ld32f(TM2 + lane_base + c0, d);
+        ld32f(TM2 + lane_base + cg0 + c0, d);
 #pragma unroll
         for (int q = 0; q < 32; ++q) {
           h[c0 + q] = fmaf(gam, h[c0 + q], d[q]);
           d[q] = h[c0 + q];
         }
-        store_brow32<NV, 128>(sH, tid, c0, d);
+        store_brow32<NV, 128>(sH, row, cg0 + c0, d);
       }
       fence_proxy_async_smem();
       tc_fence_before_sync();
-      named_arrive(BAR_H_READY, 128 + 32);
+      named_arrive(BAR_H_READY, NCOMP + 32);
       HA_PROF(chain, 8 * c + 5);
     }
 
     if (p.hT) {
-      const size_t base = (((size_t)n * p.HV + j) * 128 + tid) * 128 + (size_t)slice * NV;
+      const size_t base = (((size_t)n * p.HV + j) * 128 + row) * 128 + (size_t)slice * NV + cg0;
 #pragma unroll
-      for (int q = 0; q < NV; q += 4)
+      for (int q = 0; q < NVT; q += 4)
         *reinterpret_cast<float4*>(p.hT + base + q) = make_float4(h[q], h[q + 1], h[q + 2], h[q + 3]);
     }
   }
 
-  if (warp == 5) named_sync(BAR_H_READY, 128 + 32);      // pairs with the compute warps' last arrival
+  if (warp == W_MMA) named_sync(BAR_H_READY, NCOMP + 32);  // pairs with the compute warps' last arrival
   if (*abort_flag && tid == 0) report_status(p.status, HA_LA_ERR_TIMEOUT);
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
 }
 
-template <int NV, bool KDA, int S>
+template <int NV, bool KDA, int S, int CG>
 cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, int grid, cudaStream_t stream) {
-  auto kern = tc_chain_kernel<NV, KDA, S>;
+  auto kern = tc_chain_kernel<NV, KDA, S, CG>;
   constexpr int smem = ChainCfg<NV, S>::kSmem;
   static_assert(smem <= 227 * 1024, "shared memory budget");
   if (!cp) {                                             // configure only (this also loads the kernel)
@@ -352,22 +359,19 @@ cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, int grid, cudaS
     return cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
   }
   timer_mark(stream, "tc_chain");
-  kern<<<grid, kChainThreads, smem, stream>>>(*mk, *cp);
+  kern<<<grid, chain_threads(CG), smem, stream>>>(*mk, *cp);
   return cudaGetLastError();
 }
 
+// Slices of 64 and 128 value channels are worked on by two column groups of compute warps.
 template <bool KDA>
-cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, int nv, bool two_stage, int grid,
-                        cudaStream_t stream) {
-  if (nv == 32) return two_stage ? run_nv<32, KDA, 2>(cp, mk, grid, stream) : run_nv<32, KDA, 3>(cp, mk, grid, stream);
-  if (nv == 64) return two_stage ? run_nv<64, KDA, 2>(cp, mk, grid, stream) : run_nv<64, KDA, 3>(cp, mk, grid, stream);
-  return run_nv<128, KDA, 2>(cp, mk, grid, stream);
+cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, int nv, int grid, cudaStream_t stream) {
+  if (nv == 32) return run_nv<32, KDA, 3, 1>(cp, mk, grid, stream);
+  if (nv == 64) return run_nv<64, KDA, 3, 2>(cp, mk, grid, stream);
+  return run_nv<128, KDA, 2, 2>(cp, mk, grid, stream);
 }
 
 }  // namespace
-
-// Shared memory of the two-stage NV = 32 chain CTA: with it, one chain CTA and one prep CTA fit on an SM.
-size_t tc_chain_smem_two_stage_nv32() { return ChainCfg<32, 2>::kSmem; }
 
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                             const CUtensorMap& mk, int nv, int32_t epoch, cudaStream_t stream) {
@@ -379,15 +383,14 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   cp.epoch = epoch;
   const int grid = p.N * p.HV * (128 / nv);
   if (grid == 0) return cudaSuccess;
-  const bool two_stage = false;                          // three stages also keep prep CTAs off the chain's SMs
-  return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, nv, two_stage, grid, stream)
-                                : run_variant<false>(&cp, &mk, nv, two_stage, grid, stream);
+  return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, nv, grid, stream)
+                                : run_variant<false>(&cp, &mk, nv, grid, stream);
 }
 
 // Attributes (and loading) of the chain kernel instance a launch will use; see configure_tc_prep.
-cudaError_t configure_tc_chain(const Problem& p, int nv, bool concurrent) {
-  return p.variant == HA_LA_KDA ? run_variant<true>(nullptr, nullptr, nv, concurrent, 0, nullptr)
-                                : run_variant<false>(nullptr, nullptr, nv, concurrent, 0, nullptr);
+cudaError_t configure_tc_chain(const Problem& p, int nv) {
+  return p.variant == HA_LA_KDA ? run_variant<true>(nullptr, nullptr, nv, 0, nullptr)
+                                : run_variant<false>(nullptr, nullptr, nv, 0, nullptr);
 }
 
 }  // namespace ha_la

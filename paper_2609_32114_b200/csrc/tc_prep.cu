@@ -53,7 +53,8 @@ constexpr uint32_t OFF_TU = OFF_R1 + 8192;
 constexpr uint32_t OFF_WT = OFF_R1;                      // bf16 [128][64] K-major, swizzled (16 KiB)
 constexpr uint32_t OFF_P = OFF_R1 + 16384;               // bf16 [64][64] K-major, swizzled
 constexpr uint32_t OFF_MISC = OFF_P + 8192;              // floats: G[64], beta[64], e^G[64], beta e^G[64], G log2e[64]
-constexpr uint32_t OFF_BAR = OFF_MISC + 5 * 64 * 4;
+constexpr uint32_t OFF_RAW = OFF_MISC + 5 * 64 * 4;      // floats: log-gate[64], beta[64] of the NEXT item (cp.async)
+constexpr uint32_t OFF_BAR = OFF_RAW + 2 * 64 * 4;
 constexpr uint32_t kPrepSmem = OFF_BAR + 64;
 static_assert(OFF_D + 4 * 256 * 2 <= OFF_P, "solve scratch overlaps P");
 static_assert(3 * (kPrepSmem + 1024) <= 228 * 1024, "three CTAs per SM");
@@ -90,6 +91,11 @@ __device__ __forceinline__ void ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+
+__device__ __forceinline__ void cp_async4(void* sdst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(sdst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 __device__ __forceinline__ float ex2(float x) {          // 2^x, flushes to zero for very negative x
   float y;
@@ -214,12 +220,13 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   float* sBeta = sG + 64;
   float* sEG = sG + 128;
   float* sBE = sG + 192;
+  float* sRaw = reinterpret_cast<float*>(sm + OFF_RAW);
   uint64_t* bar_load = reinterpret_cast<uint64_t*>(sm + OFF_BAR);
   uint64_t* bar_mma = bar_load + 1;
   uint64_t* bar_v = bar_load + 2;                        // the V tiles arrive on their own barrier
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_load + 3);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* sTmp = reinterpret_cast<float*>(tmem_slot + 2);
+  int* sNext = reinterpret_cast<int*>(tmem_slot + 2);    // next item: have, j, jq, L, tok0 (written by thread 0)
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
@@ -229,7 +236,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
   HA_PROF(prep, 0);
   HA_PROF_SMID(prep, 256, 512);
-#define PP(slot) do { if (cjl == (long long)gridDim.x) HA_PROF(prep, slot); } while (0)
+#define PP(slot) HA_PROF(prep, 16 + 16 * (int)(cjl / gridDim.x) + (slot))
 
   if (tid == 0) {
     mbar_init(bar_load, 1);
@@ -254,9 +261,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   uint32_t mph = 0;                                      // parity of the next MMA-completion wait
   uint32_t lph = 0;                                      // parity of the next tile-load wait
   long long prev_cj = -1;                                // item whose bulk stores are still in flight (thread 0)
-  auto item_geom = [&](long long c, int& j_, int& jq_, int& L_, int& tok0_) {
-    const int s_ = (int)(c / p.HV);
-    j_ = (int)(c % p.HV);
+  auto item_geom = [&](long long c, int& j_, int& jq_, int& L_, int& tok0_) {   // (the item count fits 31 bits)
+    const int s_ = (int)((unsigned)c / (unsigned)p.HV);
+    j_ = (int)((unsigned)c - (unsigned)s_ * (unsigned)p.HV);
     jq_ = j_ / (p.HV / p.HK);
     if (p.chunk_len) {
       L_ = p.chunk_len[s_];
@@ -290,23 +297,36 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   int j = 0, jq = 0, L = 0, tok0 = 0;
   bool have = cjl < p.total;
   if (have) { item_geom(cjl, j, jq, L, tok0); have = L > 0; }   // unused chunk slots come last
-  float g_pre = 0.f, b_pre = 0.f;                        // GDN, threads 0..63: this token's log-gate and beta
+  // GDN: warp 1 stages the log-gates and betas of an item in shared memory with cp.async (two tokens per lane),
+  // one item ahead, and scans them at the top of that item.
+  auto stage_gates = [&](int j_, int L_, int tok0_) {
+    if (!KDA && warp == 1) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int t = lane + 32 * h;
+        if (t < L_) {
+          cp_async4(sRaw + t, p.g + (size_t)(tok0_ + t) * p.HV + j_);
+          cp_async4(sRaw + 64 + t, p.beta + (size_t)(tok0_ + t) * p.HV + j_);
+        } else {
+          sRaw[t] = 0.f;
+          sRaw[64 + t] = 0.f;
+        }
+      }
+    }
+  };
   if (have) {
     if (tid == 0) issue_tiles(jq, tok0);
-    if (!KDA && tid < L && tid < 64) {
-      g_pre = p.g[(size_t)(tok0 + tid) * p.HV + j];
-      b_pre = p.beta[(size_t)(tok0 + tid) * p.HV + j];
-    }
+    stage_gates(j, L, tok0);
   }
   while (have) {
   const size_t cj = (size_t)cjl;
-  // The previous item's bulk stores must have read their shared-memory sources before anything is overwritten.
-  if (tid == 0) {
-    if (prev_cj >= 0) bulk_wait_read_all();
-    issue_v(j, tok0);                                    // lands where the previous item's O_loc image was
-  }
-  __syncthreads();
   if constexpr (KDA) {
+    // The previous item's bulk stores must have read their shared-memory sources before anything is overwritten.
+    if (tid == 0) {
+      if (prev_cj >= 0) bulk_wait_read_all();
+      issue_v(j, tok0);
+    }
+    __syncthreads();
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
     float* sGc = reinterpret_cast<float*>(sm + OFF_G);
     {
@@ -498,27 +518,24 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
   } else {
-    // ---- op #1 Gate: inclusive scan of the log-gate over the chunk (threads 0..63)
-    if (tid < 64) {
-      float x = g_pre;                                   // fetched while the previous item was finishing
-      const float b = b_pre;
+    // ---- op #1 Gate: inclusive scan of the log-gate over the chunk (warp 1, tokens lane and lane + 32)
+    if (warp == 1) {
+      cp_async_wait_all();
+      float x0 = sRaw[lane], x1 = sRaw[lane + 32];
+      const float b0 = sRaw[64 + lane], b1 = sRaw[96 + lane];
   #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const float y = __shfl_up_sync(0xffffffffu, x, o);
-        if (lane >= o) x += y;
+        const float y0 = __shfl_up_sync(0xffffffffu, x0, o), y1 = __shfl_up_sync(0xffffffffu, x1, o);
+        if (lane >= o) { x0 += y0; x1 += y1; }
       }
-      if (tid == 31) *sTmp = x;
-      sBeta[tid] = b;
-      sG[tid] = x;                                         // warp 1 adds warp 0's total below
-    }
-    __syncthreads();
-    if (tid >= 32 && tid < 64) sG[tid] += *sTmp;
-    __syncthreads();
-    if (tid < 64) {
-      const float e = __expf(sG[tid]);
-      sEG[tid] = e;
-      sBE[tid] = e * sBeta[tid];
-      sBE[64 + tid] = sG[tid] * 1.4426950408889634f;      // G log2(e), for ex2 in the decay mask
+      x1 += __shfl_sync(0xffffffffu, x0, 31);
+      const float e0 = __expf(x0), e1 = __expf(x1);
+      sG[lane] = x0;             sG[lane + 32] = x1;
+      sBeta[lane] = b0;          sBeta[lane + 32] = b1;
+      sEG[lane] = e0;            sEG[lane + 32] = e1;
+      sBE[lane] = e0 * b0;       sBE[lane + 32] = e1 * b1;
+      sBE[64 + lane] = x0 * 1.4426950408889634f;           // G log2(e), for ex2 in the decay mask
+      sBE[96 + lane] = x1 * 1.4426950408889634f;
     }
 
     // ---- op #2 KKT (+ Q K^T): S[0:64] = K K^T, S[64:128] = Q K^T
@@ -526,6 +543,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       PP(2);
       mbar_wait(bar_load, lph, abort_flag);
       PP(3);
+      // the previous item's W / U images must have left before V lands on one and A is written over the other
+      if (prev_cj >= 0) bulk_wait_read_all();
+      issue_v(j, tok0);
       tc_fence_after_sync();
       const uint32_t id = idesc_bf16(128, 64, false, false);
       const uint32_t base = smem_u32(sm + OFF_KQ);
@@ -718,8 +738,11 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       umma_ss(tmem + 64, smem_desc(smem_u32(sm + OFF_UT) + ks * 32, 16, 1024, kSwizzle128B),
               smem_desc(smem_u32(sm + OFF_P) + ks * 32, 16, 1024, kSwizzle128B), id, ks > 0);
     umma_commit(bar_mma);
+    // two bulk groups, so that the Q~ image can follow the W image before the U image has been read too
     bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes, sm + OFF_WT, kImgBytes);
+    bulk_commit();
     bulk_store(p.ws.u + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
+    if constexpr (KDA) bulk_store(p.ws.kd + (size_t)cj * kImgBytes, sm + OFF_KD, kImgBytes);
     bulk_commit();
   }
   if (tid >= 64) {                                       // per-chunk scalars for the chain kernel
@@ -733,7 +756,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
   }
   if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
-  if (tid == 0) bulk_wait_read_all();                    // the W^T / U^T tiles were read; they receive the next images
+  if (tid == 0) bulk_wait_read_1();                      // the W image was read; it receives the Q~ image
   mph ^= 1;
   __syncthreads();
   PP(12);
@@ -741,38 +764,46 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // Every MMA of this item is done, so the K / Q tile regions are free: start the next item's loads now
   // (its V tiles follow at the top of the loop, once the O_loc image has left their room).
   const long long nxt = cjl + gridDim.x;
-  int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
-  bool have_n = nxt < p.total;
-  if (have_n) { item_geom(nxt, jn, jqn, Ln, tok0n); have_n = Ln > 0; }
-  float g_n = 0.f, b_n = 0.f;
-  if (have_n) {
-    if (tid == 0) issue_tiles(jqn, tok0n);
-    if (!KDA && tid < Ln && tid < 64) {
-      g_n = p.g[(size_t)(tok0n + tid) * p.HV + jn];
-      b_n = p.beta[(size_t)(tok0n + tid) * p.HV + jn];
-    }
+  if (tid == 0) {                                        // one thread works out where the next item is
+    int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
+    bool hn = nxt < p.total;
+    if (hn) { item_geom(nxt, jn, jqn, Ln, tok0n); hn = Ln > 0; }
+    PP(14);
+    if (hn) issue_tiles(jqn, tok0n);
+    PP(15);
+    sNext[0] = hn ? 1 : 0; sNext[1] = jn; sNext[2] = jqn; sNext[3] = Ln; sNext[4] = tok0n;
   }
   {
     // Q~^T and O_loc^T are complete in the accumulators; their images go where W^T and U^T were.
     float v[32];
     ld32(my_tmem, v);
     store_half_row(v, rowq, hf, sm + OFF_WT);
+    if (tid == 0) bulk_wait_read_all();                  // the U image was read too
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_WT, kImgBytes);
+      bulk_commit();
+    }
+    if (sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4]);
     ld32(my_tmem + 64, v);
     store_half_row(v, rowq, hf, sm + OFF_UT);
   }
+  // The accumulators were read: the next item's first MMA may overwrite them after this barrier.
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
   if (tid == 0) {
-    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_WT, kImgBytes);
     bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
-    if constexpr (KDA) bulk_store(p.ws.kd + (size_t)cj * kImgBytes, sm + OFF_KD, kImgBytes);
     bulk_commit();
   }
+  const bool have_n = sNext[0] != 0;
+  const int jn = sNext[1], jqn = sNext[2], Ln = sNext[3], tok0n = sNext[4];
+  PP(13);
   prev_cj = cjl;
   lph ^= 1;
-  cjl = nxt; have = have_n; j = jn; jq = jqn; L = Ln; tok0 = tok0n; g_pre = g_n; b_pre = b_n;
-  PP(13);
+  cjl = nxt; have = have_n; j = jn; jq = jqn; L = Ln; tok0 = tok0n;
   }  // work items
 
   __syncthreads();
