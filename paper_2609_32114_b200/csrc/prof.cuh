@@ -7,10 +7,14 @@
   extern "C" int ha_la_debug_read_prof_##name(long long* out) {                                   \
     return cudaMemcpyFromSymbol(out, g_prof_##name, sizeof(long long) * 1024) == cudaSuccess ? 0 : 4; \
   }
+#ifdef HA_LA_PROFILE_COARSE
+#define HA_PROF(name, slot) do { } while (0)
+#else
 #define HA_PROF(name, slot)                                                            \
   do {                                                                                 \
     if (threadIdx.x == 0 && blockIdx.x == 0 && (slot) < 1024) g_prof_##name[slot] = clock64(); \
   } while (0)
+#endif
 // records the SM id of CTA `blockIdx.x` at slot base + blockIdx.x % count
 #define HA_PROF_SMID(name, base, count)                                                \
   do {                                                                                 \
@@ -20,7 +24,15 @@
       g_prof_##name[(base) + blockIdx.x % (count)] = smid_;                            \
     }                                                                                  \
   } while (0)
+// stores the global nanosecond timer at `slot` (any CTA; the caller picks who records)
+#define HA_PROF_GT(name, slot)                                                         \
+  do {                                                                                 \
+    unsigned long long gt_;                                                            \
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_));                            \
+    if ((slot) >= 0 && (slot) < 1024) g_prof_##name[slot] = (long long)gt_;            \
+  } while (0)
 #else
+#define HA_PROF_GT(name, slot) do { } while (0)
 #define HA_PROF_SMID(name, base, count) do { } while (0)
 #define HA_PROF_DECL(name)
 #define HA_PROF(name, slot) do { } while (0)

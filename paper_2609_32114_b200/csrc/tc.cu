@@ -1,19 +1,18 @@
 // Tensor-core (tcgen05) path, host side: tensor maps, workspace carving, slice-width choice, launches.
 //
-// Two launch modes.  Sequential: prep kernel, then chain kernel, both on the caller's stream.
-// Concurrent: the prep kernel runs on an internal stream next to the chain kernel, which
-// consumes each chunk as soon as the prep CTA of that chunk has published it (release/acquire flag
-// per chunk in the workspace, stamped with a per-call epoch so that nothing has to be cleared).  The
-// internal stream forks from and joins back into the caller's stream with two events, so the call
-// stays asynchronous and ordered like any other work on that stream.  The concurrent mode is opt-in
-// (HA_LA_TC_OVERLAP=1) and only used when the chain CTAs leave SMs free (at most one chain CTA per two
-// SMs); the persistent prep kernel is then sized to the free SMs.  Its first use on a device creates the
-// internal stream and events and should not happen inside a stream capture.
+// Both kernels go on the caller's stream; the chain kernel is launched as a programmatic dependent of the
+// prep kernel, so it may start once every prep CTA is running.  Two modes:
+//   sequential: the chain kernel sets itself up under the prep kernel's tail and then waits for that whole grid;
+//   concurrent: when the chain CTAs need at most half of the SMs, the prep kernel is sized to the other SMs
+//     (one CTA per SM) and the chain kernel consumes each chunk as soon as the prep work group of that chunk
+//     has published it (release/acquire flag per chunk in the workspace, stamped with a per-call epoch so that
+//     nothing has to be cleared).  The flags' producer is running (or done) before a consumer starts, whatever
+//     else the GPU is doing, so the consumer's bounded waits cannot starve.
+// HA_LA_TC_OVERLAP=0 forces the sequential mode.
 #include <cuda.h>
 #include <stdlib.h>
 
 #include <atomic>
-#include <mutex>
 
 #include "tc_common.cuh"
 
@@ -23,7 +22,7 @@ cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanVi
                            const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int32_t epoch,
                            int reserved_sms, cudaStream_t stream);
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                            const CUtensorMap& mk, int nv, int32_t epoch, cudaStream_t stream);
+                            const CUtensorMap& mk, int nv, int32_t epoch, bool dependent, cudaStream_t stream);
 
 cudaError_t configure_tc_prep(const Problem& p);
 cudaError_t configure_tc_chain(const Problem& p, int nv);
@@ -82,43 +81,14 @@ int pick_nv(const Problem& p) {
   return 128;
 }
 
-// Per-device side stream and fork/join events of the concurrent mode, created on first use.
-struct SideStream {
-  cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
-  bool tried = false, ok = false;
-};
-constexpr int kMaxDevices = 64;
-SideStream g_side[kMaxDevices];
 std::atomic<int32_t> g_epoch{0};
-
-SideStream* side_stream() {
-  static std::mutex mu;
-  std::lock_guard<std::mutex> lock(mu);
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-  SideStream& s = g_side[dev];
-  if (!s.tried) {
-    s.tried = true;
-    int least = 0, greatest = 0;
-    if (cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess &&
-        cudaStreamCreateWithPriority(&s.stream, cudaStreamNonBlocking, least) == cudaSuccess &&
-        cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) == cudaSuccess &&
-        cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) == cudaSuccess)
-      s.ok = true;
-  }
-  return s.ok ? &s : nullptr;
-}
 
 bool want_concurrent(const Problem& p, int nv) {
   if (g_timer) return false;                             // per-kernel timing wants one kernel at a time
-  // Opt-in: the chain kernel then spins (bounded) on flags that the prep kernel publishes, which needs the
-  // prep kernel to get SMs of its own; when other streams oversubscribe the GPU a wait could run out
-  // and the call would report HA_LA_ERR_TIMEOUT.  Measured gain on the headline workload: about 3 %.
   const char* e = getenv("HA_LA_TC_OVERLAP");
-  if (!e || e[0] != '1') return false;
+  if (e && e[0] == '0') return false;
   const long long chain_ctas = (long long)p.N * p.HV * (128 / nv);
-  return nv <= 64 && chain_ctas * 2 <= sm_count() && p.max_chunks > 1;
+  return chain_ctas * 2 <= sm_count() && p.max_chunks > 1;
 }
 
 }  // namespace
@@ -141,34 +111,23 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
   const int nv = pick_nv(p);
 
-  SideStream* side = want_concurrent(p, nv) ? side_stream() : nullptr;
-  // Configure (and load) both kernels before anything is enqueued.
+  const bool concurrent = want_concurrent(p, nv);
+  // Configure (and load) both kernels before anything is enqueued: loading a kernel for the first time can
+  // wait for the device, and in the concurrent mode the chain kernel would be spinning meanwhile.
   cudaError_t ce = configure_tc_prep(p);
   if (ce != cudaSuccess) return ce;
   ce = configure_tc_chain(p, nv);
   if (ce != cudaSuccess) return ce;
-  if (!side) {
-    cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, 0, 0, stream);
-    if (e != cudaSuccess) return e;
-    return launch_tc_chain(p, a, plan, ws, mk, nv, 0, stream);
+  int32_t epoch = 0;                                     // 0 means "sequential"
+  int reserved_sms = 0;
+  if (concurrent) {
+    epoch = g_epoch.fetch_add(1) + 1;
+    if (epoch == 0) epoch = g_epoch.fetch_add(1) + 1;
+    reserved_sms = p.N * p.HV * (128 / nv);              // a chain CTA fills its SM
   }
-
-  int32_t epoch = g_epoch.fetch_add(1) + 1;
-  if (epoch == 0) epoch = g_epoch.fetch_add(1) + 1;      // 0 means "sequential"
-  cudaError_t e = cudaEventRecord(side->fork, stream);
+  cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, reserved_sms, stream);
   if (e != cudaSuccess) return e;
-  e = cudaStreamWaitEvent(side->stream, side->fork, 0);
-  if (e != cudaSuccess) return e;
-  // The chain kernel goes on the caller's stream and is enqueued first, so that its CTAs are resident (one
-  // per SM) before the prep CTAs arrive; the prep kernel runs on the side stream and fills the remaining room.
-  e = launch_tc_chain(p, a, plan, ws, mk, nv, epoch, stream);
-  if (e != cudaSuccess) return e;
-  // a chain CTA (three stages) fills its SM: the prep kernel gets the other SMs
-  e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, p.N * p.HV * (128 / nv), side->stream);
-  if (e != cudaSuccess) return e;
-  e = cudaEventRecord(side->join, side->stream);
-  if (e != cudaSuccess) return e;
-  return cudaStreamWaitEvent(stream, side->join, 0);
+  return launch_tc_chain(p, a, plan, ws, mk, nv, epoch, /*dependent=*/g_timer == nullptr, stream);
 }
 
 }  // namespace ha_la

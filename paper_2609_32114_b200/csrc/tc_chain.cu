@@ -67,6 +67,7 @@ struct ChainParams {
   int HK, HV;
   float scale;
   int32_t epoch;               // != 0: the prep kernel runs concurrently; wait for ws.flags[cj] == epoch per chunk
+                               // == 0: wait for the whole prep grid before the first workspace read
   int32_t* status;
 };
 
@@ -153,7 +154,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   const int chunk0 = p.seq_tok0 ? p.seq_chunk0[n] : n * p.cps;
   const int nchunks = (len + kChunk - 1) / kChunk;
 
-  HA_PROF_SMID(chain, 768, 128);
+  if (blockIdx.x == 0 && threadIdx.x == 0) HA_PROF_GT(chain, 900);
   if (tid == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], NCOMP); }
     mbar_init(bar_mma1, 1);
@@ -168,26 +169,44 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
   const uint32_t TM1 = tmem, TM2 = tmem + NV;
+  // This kernel may be launched as a programmatic dependent of the prep kernel, i.e. start while that one is
+  // still running.  Sequential mode: everything above overlapped the prep kernel's tail; wait for it here.
+  if (p.epoch == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
   uint8_t* sH = sm + Cfg::OFF_H;
   uint8_t* sUt = sm + Cfg::OFF_UT;
 
   if (warp == W_PROD) {
     // ------------------------------------------------------------ producer
-    if ((tid & 31) == 0) {
-      for (int c = 0; c < nchunks; ++c) {
+    // Concurrent mode: the whole warp looks at the ready flags of the next 32 chunks at once (plain loads) and
+    // remembers how far the prep kernel has got; the acquire fence and the proxy fence, which are what makes
+    // the published images visible to this kernel's bulk copies, are then paid once per batch, not per chunk.
+    const int lane = tid & 31;
+    int ready_upto = p.epoch != 0 ? 0 : nchunks;         // chunks [0, ready_upto) are known to be published
+    for (int c = 0; c < nchunks; ++c) {
+      if (c >= ready_upto) {
+        int got = 0;
+        for (uint32_t it = 0; it < kSpinLimit && !*abort_flag; ++it) {
+          const int cc = c + lane;
+          bool ok = false;
+          if (cc < nchunks)
+            ok = *reinterpret_cast<const volatile int32_t*>(p.ws.flags + (size_t)(chunk0 + cc) * p.HV + j) == p.epoch;
+          const unsigned m = __ballot_sync(0xffffffffu, ok);
+          got = __ffs(~m) - 1;                           // leading published chunks (32 when all are)
+          if (got < 0) got = 32;
+          if (got > 0) break;
+          __nanosleep(100);
+        }
+        if (got == 0) *abort_flag = 1;                   // gave up: carry on, the status word reports the time-out
+        ready_upto = c + (got > 0 ? got : nchunks);
+        __threadfence();                                 // acquire side of the prep kernel's release
+        fence_proxy_async_all();
+        if (blockIdx.x == 0 && lane == 0) HA_PROF_GT(chain, 600 + c);
+      }
+      if (lane == 0) {
         const int st = c % S;
         if (c >= S) mbar_wait(&bar_empty[st], ((c / S) - 1) & 1, abort_flag);
         uint8_t* stage = sm + st * Cfg::kStageB;
         const size_t cj = (size_t)(chunk0 + c) * p.HV + j;
-        if (p.epoch != 0) {                              // bounded wait for the prep CTA of this chunk
-          bool ready = false;
-          for (uint32_t it = 0; it < kSpinLimit && !*abort_flag; ++it) {
-            if (ld_acquire_gpu(p.ws.flags + cj) == p.epoch) { ready = true; break; }
-            __nanosleep(40);
-          }
-          if (!ready) *abort_flag = 1;
-          fence_proxy_async_all();
-        }
         mbar_expect_tx(&bar_full[st], Cfg::kTxBytes);
         bulk_load(stage + Cfg::OFF_WQ, p.ws.wq + cj * 2 * kImgBytes, 32768, &bar_full[st]);
         bulk_load(stage + Cfg::OFF_U, p.ws.u + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
@@ -200,6 +219,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
           tma_load_3d(stage + Cfg::OFF_K + 8192, &map_k, &bar_full[st], 64, jq, tok0 + c * kChunk);
         }
       }
+      __syncwarp();
     }
   } else if (warp == W_MMA) {
     // ------------------------------------------------------------ MMA issue (lane 0 issues; the warp keeps the barriers)
@@ -331,6 +351,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
       tc_fence_before_sync();
       named_arrive(BAR_H_READY, NCOMP + 32);
       HA_PROF(chain, 8 * c + 5);
+      if (blockIdx.x == 0 && tid == 0 && (c == 0 || c == nchunks - 1)) HA_PROF_GT(chain, 700 + c);
     }
 
     if (p.hT) {
@@ -343,13 +364,17 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
 
   if (warp == W_MMA) named_sync(BAR_H_READY, NCOMP + 32);  // pairs with the compute warps' last arrival
   if (*abort_flag && tid == 0) report_status(p.status, HA_LA_ERR_TIMEOUT);
+  // Concurrent mode: do not finish before the prep grid has (it has published its last chunk by now), so that
+  // work queued behind this kernel is also behind the prep kernel.
+  if (p.epoch != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
   tc_fence_before_sync();
   __syncthreads();
+  if (threadIdx.x == 0) HA_PROF_GT(chain, 901);
   if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
 }
 
 template <int NV, bool KDA, int S, int CG>
-cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, int grid, cudaStream_t stream) {
+cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, int grid, bool dependent, cudaStream_t stream) {
   auto kern = tc_chain_kernel<NV, KDA, S, CG>;
   constexpr int smem = ChainCfg<NV, S>::kSmem;
   static_assert(smem <= 227 * 1024, "shared memory budget");
@@ -359,22 +384,34 @@ cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, int grid, cudaS
     return cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
   }
   timer_mark(stream, "tc_chain");
-  kern<<<grid, chain_threads(CG), smem, stream>>>(*mk, *cp);
-  return cudaGetLastError();
+  // `dependent`: programmatic dependent launch behind the prep kernel (same stream): the CTAs may start as soon
+  // as every prep CTA is running, instead of after the prep grid has drained.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(chain_threads(CG));
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, *mk, *cp);
 }
 
 // Slices of 64 and 128 value channels are worked on by two column groups of compute warps.
 template <bool KDA>
-cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, int nv, int grid, cudaStream_t stream) {
-  if (nv == 32) return run_nv<32, KDA, 3, 1>(cp, mk, grid, stream);
-  if (nv == 64) return run_nv<64, KDA, 3, 2>(cp, mk, grid, stream);
-  return run_nv<128, KDA, 2, 2>(cp, mk, grid, stream);
+cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, int nv, int grid, bool dependent,
+                        cudaStream_t stream) {
+  if (nv == 32) return run_nv<32, KDA, 3, 1>(cp, mk, grid, dependent, stream);
+  if (nv == 64) return run_nv<64, KDA, 3, 2>(cp, mk, grid, dependent, stream);
+  return run_nv<128, KDA, 2, 2>(cp, mk, grid, dependent, stream);
 }
 
 }  // namespace
 
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                            const CUtensorMap& mk, int nv, int32_t epoch, cudaStream_t stream) {
+                            const CUtensorMap& mk, int nv, int32_t epoch, bool dependent, cudaStream_t stream) {
   ChainParams cp;
   cp.h0 = a.h0; cp.hT = a.hT; cp.o = a.o;
   cp.seq_tok0 = plan.seq_tok0; cp.seq_len = plan.seq_len; cp.seq_chunk0 = plan.seq_chunk0;
@@ -383,14 +420,14 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   cp.epoch = epoch;
   const int grid = p.N * p.HV * (128 / nv);
   if (grid == 0) return cudaSuccess;
-  return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, nv, grid, stream)
-                                : run_variant<false>(&cp, &mk, nv, grid, stream);
+  return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, nv, grid, dependent, stream)
+                                : run_variant<false>(&cp, &mk, nv, grid, dependent, stream);
 }
 
 // Attributes (and loading) of the chain kernel instance a launch will use; see configure_tc_prep.
 cudaError_t configure_tc_chain(const Problem& p, int nv) {
-  return p.variant == HA_LA_KDA ? run_variant<true>(nullptr, nullptr, nv, 0, nullptr)
-                                : run_variant<false>(nullptr, nullptr, nv, 0, nullptr);
+  return p.variant == HA_LA_KDA ? run_variant<true>(nullptr, nullptr, nv, 0, false, nullptr)
+                                : run_variant<false>(nullptr, nullptr, nv, 0, false, nullptr);
 }
 
 }  // namespace ha_la

@@ -37,7 +37,7 @@ HA_PROF_DECL(prep)
 
 namespace {
 
-constexpr int kPrepThreads = 256;
+constexpr int kPrepThreads = 256;        // threads of one work group (a CTA holds kGroups of them)
 constexpr int LDH = 72;                  // row stride (halfs) of the fp16 64x64 matrix A / T
 
 // shared-memory map (bytes from the 1024-aligned base); 73.3 KiB, so that three CTAs fit one SM
@@ -57,18 +57,25 @@ constexpr uint32_t OFF_RAW = OFF_MISC + 5 * 64 * 4;      // floats: log-gate[64]
 constexpr uint32_t OFF_BAR = OFF_RAW + 2 * 64 * 4;
 constexpr uint32_t kPrepSmem = OFF_BAR + 64;
 static_assert(OFF_D + 4 * 256 * 2 <= OFF_P, "solve scratch overlaps P");
-static_assert(3 * (kPrepSmem + 1024) <= 228 * 1024, "three CTAs per SM");
+// GDN: one CTA per SM holds three independent work groups (256 threads and one copy of this map each, their own
+// named barrier and quarter of tensor memory), which is the occupancy of three small CTAs but leaves whole SMs
+// to a concurrently running chain kernel.  KDA (larger map): one group.
+constexpr uint32_t kGroupSmem = (kPrepSmem + 1023) / 1024 * 1024;
+template <bool KDA> constexpr int kGroups = KDA ? 1 : 3;
+static_assert(3 * kGroupSmem <= 227 * 1024, "three work groups per CTA");
 // KDA only: per-channel cumulative log-gate (fp32, times log2 e) and the K e^{G_L - G} operand image
 constexpr int LDG = 132;                                  // row stride (floats) of the 64 x 128 gate matrix
 constexpr uint32_t OFF_G = (kPrepSmem + 1023) / 1024 * 1024;
 constexpr uint32_t OFF_KD = (OFF_G + 64 * LDG * 4 + 1023) / 1024 * 1024;   // [kb][64 tok][64 feat], like the K tile
-// K+ / Q+ rows (block b: 16 K+ rows then 16 Q+ rows; 160 rows so that an M = 64 operand may start at row 96)
-constexpr uint32_t OFF_KQP = OFF_KD + 16384;              // [kb][160 rows][128 B], K-major, swizzled
-constexpr uint32_t KQP_KB = 160 * 128;
-// K- rows for block-rows I = 1, 2, 3 (16, 32, 48 rows, starting at rows 0, 16, 48)
-constexpr uint32_t OFF_KM = OFF_KQP + 2 * KQP_KB;         // [kb][96 rows][128 B], K-major, swizzled
-constexpr uint32_t KM_KB = 96 * 128;
-constexpr uint32_t kPrepSmemKda = OFF_KM + 2 * KM_KB;
+// K+ / Q+ rows (block b: 16 K+ rows then 16 Q+ rows): one M = 128 operand
+constexpr uint32_t OFF_KQP = OFF_KD + 16384;              // [kb][128 rows][128 B], K-major, swizzled
+constexpr uint32_t KQP_KB = 128 * 128;
+// K- rows for block-rows I = 0..3 (16, 32, 48, 64 rows, starting at rows 0, 16, 48, 96)
+constexpr uint32_t OFF_KM = OFF_KQP + 2 * KQP_KB;         // [kb][160 rows][128 B], K-major, swizzled
+constexpr uint32_t KM_KB = 160 * 128;
+constexpr uint32_t OFF_FALL = OFF_KM + 2 * KM_KB;         // int[4]: diagonal block needs the element-wise evaluation
+constexpr uint32_t kPrepSmemKda = OFF_FALL + 16;
+constexpr float kMaxUpExp = 100.f;                        // largest exponent (base 2) allowed in a K- factor
 static_assert(kPrepSmemKda <= 227 * 1024, "KDA shared memory budget");
 
 struct PrepParams {
@@ -209,11 +216,17 @@ __device__ __forceinline__ void store_half_row(const float (&v)[32], int row, in
 }
 
 template <bool KDA>
-__global__ void __launch_bounds__(kPrepThreads, KDA ? 1 : 3)
+__global__ void __launch_bounds__(kPrepThreads * kGroups<KDA>, 1)
 tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, PrepParams p) {
-  extern __shared__ __align__(1024) uint8_t smem_raw[];
-  uint8_t* sm = smem_raw;                                // no static shared memory in this kernel: 1024-aligned
+  constexpr int G = kGroups<KDA>;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];  // no static shared memory in this kernel: 1024-aligned
+  const int grp = threadIdx.x / kPrepThreads;            // work group of this thread
+  uint8_t* sm = smem_raw + grp * kGroupSmem;
+  auto gsync = [&]() {                                   // barrier of one work group
+    if (G == 1) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "r"(kPrepThreads) : "memory");
+  };
   __half* sAh = reinterpret_cast<__half*>(sm + OFF_A);  // A, then T in place
   __half* sD = reinterpret_cast<__half*>(sm + OFF_D);
   float* sG = reinterpret_cast<float*>(sm + OFF_MISC);
@@ -228,15 +241,15 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* sNext = reinterpret_cast<int*>(tmem_slot + 2);    // next item: have, j, jq, L, tok0 (written by thread 0)
 
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x % kPrepThreads;
   const int warp = tid >> 5, lane = tid & 31;
-  if (smem_u32(sm) & 1023u) {                            // the swizzled layouts need it; never seen to fail
+  if (smem_u32(smem_raw) & 1023u) {                            // the swizzled layouts need it; never seen to fail
     if (threadIdx.x == 0) report_status(p.status, HA_LA_ERR_DEVICE_CHECK);
     return;
   }
   HA_PROF(prep, 0);
-  HA_PROF_SMID(prep, 256, 512);
-#define PP(slot) HA_PROF(prep, 16 + 16 * (int)(cjl / gridDim.x) + (slot))
+  if (blockIdx.x == 0 && threadIdx.x == 0) HA_PROF_GT(prep, 900);
+#define PP(slot) HA_PROF(prep, 16 + 16 * (int)(cjl / vstride) + (slot))
 
   if (tid == 0) {
     mbar_init(bar_load, 1);
@@ -246,17 +259,22 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     mbar_fence_init();
     prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
   }
-  if (warp == 0) tmem_alloc(tmem_slot, 128);
+  // the CTA's first warp allocates tensor memory for all groups (a power of two: everything, for three groups)
+  if (threadIdx.x < 32) tmem_alloc(reinterpret_cast<uint32_t*>(smem_raw + OFF_BAR + 24), G == 1 ? 256 : 512);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem = *tmem_slot;
+  // Every CTA of this grid is running now: a dependent launch (the chain kernel) may be scheduled.  It either
+  // waits for this grid to finish or consumes chunks as they are published.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const uint32_t tmem_cta = *reinterpret_cast<const uint32_t*>(smem_raw + OFF_BAR + 24);
+  const uint32_t tmem = tmem_cta + grp * 128;
   const int rowq = (warp & 3) * 32 + lane;               // accumulator row owned by this thread
   const int hf = warp >> 2;                              // which 32 of the 64 columns
   const uint32_t my_tmem = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16) + hf * 32;
   HA_PROF(prep, 1);
 
-  // Persistent CTA: work items (chunk slot, V-head) blockIdx.x, blockIdx.x + gridDim.x, ... in that order, so
+  // Persistent groups: work items (chunk slot, V-head) g, g + #groups, ... for group g of the grid, so
   // that early chunks are finished first (the chain kernel may be consuming them concurrently).
   uint32_t mph = 0;                                      // parity of the next MMA-completion wait
   uint32_t lph = 0;                                      // parity of the next tile-load wait
@@ -291,9 +309,14 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       fence_proxy_async_all();
       __threadfence();
       st_release_gpu(p.ws.flags + prev_cj, p.epoch);
+      if (prev_cj % p.HV == 0) HA_PROF_GT(prep, 512 + (int)(prev_cj / p.HV));
     }
   };
-  long long cjl = blockIdx.x;
+  // The groups of a CTA start a third of an item apart, so that they are in different phases (tensor core /
+  // CUDA cores / waiting for memory) at any time instead of in lock step.
+  if (G > 1 && grp > 0) __nanosleep(2000u * grp);
+  const long long vstride = (long long)gridDim.x * G;    // work groups in the grid
+  long long cjl = (long long)grp * gridDim.x + blockIdx.x;   // group-major: a last partial round spreads over the SMs
   int j = 0, jq = 0, L = 0, tok0 = 0;
   bool have = cjl < p.total;
   if (have) { item_geom(cjl, j, jq, L, tok0); have = L > 0; }   // unused chunk slots come last
@@ -326,7 +349,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (prev_cj >= 0) bulk_wait_read_all();
       issue_v(j, tok0);
     }
-    __syncthreads();
+    gsync();
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
     float* sGc = reinterpret_cast<float*>(sm + OFF_G);
     {
@@ -345,32 +368,39 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       for (int idx = tid; idx < 64 * LDH * 2 / 16; idx += kPrepThreads) reinterpret_cast<uint4*>(sAh)[idx] = make_uint4(0, 0, 0, 0);
       for (int idx = tid; idx < 512; idx += kPrepThreads) reinterpret_cast<uint4*>(sm + OFF_P)[idx] = make_uint4(0, 0, 0, 0);
     }
-    __syncthreads();
+    gsync();
     {
       const int c = tid & 127, r0 = (tid >> 7) * 32;     // two threads per channel, 32 rows each
       float acc = 0.f;
       for (int i = 0; i < 32; ++i) { acc += sGc[(r0 + i) * LDG + c]; sGc[(r0 + i) * LDG + c] = acc; }
     }
-    __syncthreads();
+    gsync();
     if (tid >= 128) {
       const int c = tid & 127;
       const float add = sGc[31 * LDG + c];
       for (int i = 32; i < 64; ++i) sGc[i * LDG + c] += add;
     }
     mbar_wait(bar_load, lph, abort_flag);                // every thread reads the K / Q tiles below
-    __syncthreads();
+    gsync();
     PP(4);
 
     // ---- op #2 KKT and the masked Q K^T with per-channel decay:
     //   A_ij = beta_i sum_c k_ic k_jc 2^(G_ic - G_jc) (j < i),  P_ij = sum_c q_ic k_jc 2^(G_ic - G_jc) (j <= i).
-    // Tokens are grouped in blocks of 16.  For i in block I and j in an EARLIER block the decay factors through
-    // the gate R_I at the first token of block I:  2^(G_i - R_I) * 2^(R_I - G_j), both exponents <= 0, so the
-    // off-diagonal blocks are plain contractions of rescaled bf16 operands and go to the tensor cores:
+    // Tokens are grouped in blocks of 16.  For i in block-row I the decay factors through the gate R_I at the
+    // first token of block I:  2^(G_i - R_I) * 2^(R_I - G_j), so every block is a plain contraction of rescaled
+    // bf16 operands on the tensor cores:
     //   K+_i = k_i 2^(G_i - R_I), Q+_i = q_i 2^(G_i - R_I)   (one copy),   K-_j^(I) = k_j 2^(R_I - G_j)  (per block-row I).
-    // The four diagonal blocks are evaluated element-wise in fp32.
+    // The first exponent is <= 0.  The second is <= 0 for j in an earlier block; inside the diagonal block it is
+    // the decay accumulated since the start of the block, >= 0: it is clamped to kMaxUpExp, and a block where the
+    // clamp was hit (a decay of more than 2^100 within 16 tokens in some channel) is evaluated again afterwards,
+    // element by element in fp32.
+    int* sFall = reinterpret_cast<int*>(sm + OFF_FALL);
+    if (tid < 4) sFall[tid] = 0;
+    gsync();
     {
       const int i = tid >> 2, bi16 = i >> 4;
       const int row_k = 32 * bi16 + (i & 15);
+      bool clamped = false;
 #pragma unroll 1
       for (int q = 0; q < 4; ++q) {
         const int cc = (tid & 3) * 4 + q;
@@ -384,6 +414,18 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         *reinterpret_cast<float4*>(gr) = *reinterpret_cast<const float4*>(sGc + (bi16 * 16) * LDG + cc * 8);
         *reinterpret_cast<float4*>(gr + 4) = *reinterpret_cast<const float4*>(sGc + (bi16 * 16) * LDG + cc * 8 + 4);
         uint8_t* kqp = sm + OFF_KQP + (cc >> 3) * KQP_KB;
+        uint8_t* km = sm + OFF_KM + (cc >> 3) * KM_KB;
+        {                                                // K- for the token's own block-row (exponent >= 0)
+          float up[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            up[e] = gr[e] - gi[e];
+            clamped |= up[e] > kMaxUpExp;
+            t8[e] = kf[e] * ex2(fminf(up[e], kMaxUpExp));
+          }
+          const int r0 = bi16 == 0 ? 0 : (bi16 == 1 ? 16 : (bi16 == 2 ? 48 : 96));
+          *reinterpret_cast<uint4*>(km + sw128_offset(r0 + i, cc & 7)) = pack8(t8);
+        }
 #pragma unroll
         for (int e = 0; e < 8; ++e) { gr[e] = ex2(gi[e] - gr[e]); t8[e] = kf[e] * gr[e]; }
         *reinterpret_cast<uint4*>(kqp + sw128_offset(row_k, cc & 7)) = pack8(t8);
@@ -396,24 +438,25 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           *reinterpret_cast<float4*>(g2 + 4) = *reinterpret_cast<const float4*>(sGc + (I2 * 16) * LDG + cc * 8 + 4);
 #pragma unroll
           for (int e = 0; e < 8; ++e) t8[e] = kf[e] * ex2(g2[e] - gi[e]);
-          const int r0 = I2 == 1 ? 0 : (I2 == 2 ? 16 : 48);
-          *reinterpret_cast<uint4*>(sm + OFF_KM + (cc >> 3) * KM_KB + sw128_offset(r0 + i, cc & 7)) = pack8(t8);
+          const int r0 = I2 == 1 ? 16 : (I2 == 2 ? 48 : 96);
+          *reinterpret_cast<uint4*>(km + sw128_offset(r0 + i, cc & 7)) = pack8(t8);
         }
       }
+      if (clamped) sFall[bi16] = 1;
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
-    __syncthreads();
-    if (tid == 0) {                                      // block-row I: D_I[64 x 16 I] = [K+_I ; Q+_I ; ...] (K-^(I))^T
-      tc_fence_after_sync();
+    gsync();
+    if (tid == 0) {                        // block-row I: D_I[128 x 16 (I + 1)] = [all K+ / Q+ rows] (K-^(I))^T;
+      tc_fence_after_sync();               // only rows 32 I .. 32 I + 31 (K+_I, Q+_I) of D_I are used
 #pragma unroll
-      for (int I = 1; I < 4; ++I) {
-        const uint32_t id = idesc_bf16(64, 16 * I, false, false);
-        const uint32_t col = I == 1 ? 0 : (I == 2 ? 16 : 48);
+      for (int I = 0; I < 4; ++I) {
+        const uint32_t id = idesc_bf16(128, 16 * (I + 1), false, false);
+        const uint32_t col = I == 0 ? 0 : (I == 1 ? 16 : (I == 2 ? 48 : 96));
         const uint32_t r0 = col;                         // first K- row of this block-row = its column offset
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t a = smem_u32(sm + OFF_KQP) + (ks >> 2) * KQP_KB + (32 * I) * 128 + (ks & 3) * 32;
+          const uint32_t a = smem_u32(sm + OFF_KQP) + (ks >> 2) * KQP_KB + (ks & 3) * 32;
           const uint32_t bb = smem_u32(sm + OFF_KM) + (ks >> 2) * KM_KB + r0 * 128 + (ks & 3) * 32;
           umma_ss(tmem + col, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(bb, 16, 1024, kSwizzle128B), id, ks > 0);
         }
@@ -421,74 +464,73 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       umma_commit(bar_mma);
       publish_prev();
     }
-    // diagonal 16x16 blocks, element-wise (overlaps the MMAs): 4 blocks x 136 pairs (j <= i)
-    for (int pidx = tid; pidx < 4 * 136; pidx += kPrepThreads) {
-      const int blk = pidx / 136, qq = pidx % 136;
-      int il = 0;
-      while ((il + 1) * (il + 2) / 2 <= qq) ++il;
-      const int jl = qq - il * (il + 1) / 2;
-      const int i = blk * 16 + il, jj = blk * 16 + jl;
-      float kk = 0.f, qk = 0.f;
-#pragma unroll 2
-      for (int cc = 0; cc < 16; ++cc) {
-        const uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
-        float kif[8], qif[8], kjf[8], gi[8], gj[8];
-        unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(i, cc & 7)), kif);
-        unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + sw128_offset(i, cc & 7)), qif);
-        unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(jj, cc & 7)), kjf);
-        *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
-        *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
-        *reinterpret_cast<float4*>(gj) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8);
-        *reinterpret_cast<float4*>(gj + 4) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8 + 4);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float t = kjf[e] * ex2(gi[e] - gj[e]);
-          kk = fmaf(kif[e], t, kk);
-          qk = fmaf(qif[e], t, qk);
-        }
-      }
-      if (jj < i) sAh[i * LDH + jj] = __float2half_rn(sBeta[i] * kk);
-      *reinterpret_cast<__nv_bfloat16*>(sm + OFF_P + sw128_offset(i, jj >> 3) + (jj & 7) * 2) = __float2bfloat16_rn(qk);
-    }
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
     mph ^= 1;
-    __syncthreads();
+    gsync();
     tc_fence_after_sync();
-    if (warp < 2) {
-      // M = 64 accumulators: row r sits in lane (r % 16) + 32 (r / 16).  Rows 0..15 (K+ -> K K^T) are lanes
-      // 0..15 of warp 0, rows 16..31 (Q+ -> Q K^T) lanes 0..15 of warp 1; the other rows are padding.
-      const uint32_t tl = tmem + (static_cast<uint32_t>(warp * 32) << 16);
-      uint32_t r1[16], r2[32], r3a[32], r3b[16];
-      tmem_ld16(tl + 0, r1);
-      tmem_ld32(tl + 16, r2);
-      tmem_ld32(tl + 48, r3a);
-      tmem_ld16(tl + 80, r3b);
-      tmem_ld_wait();
-      if (lane < 16) {
+    {
+      // Block-row I sits in tensor-memory lanes 32 I .. 32 I + 31: lanes 0..15 the K+ rows (-> A), 16..31 the Q+
+      // rows (-> P).  Warps I and I + 4 share its 16-column pieces.
+      const int I = warp & 3, l16 = lane & 15;
+      const bool isq = lane >= 16;
+      const int i = 16 * I + l16;
+      const uint32_t col = I == 0 ? 0 : (I == 1 ? 16 : (I == 2 ? 48 : 96));
+      const uint32_t tl = tmem + (static_cast<uint32_t>(I * 32) << 16) + col;
+      const float bi = sBeta[i];
+      for (int cb = warp >> 2; cb <= I; cb += 2) {
+        uint32_t r[16];
+        tmem_ld16(tl + 16 * cb, r);
+        tmem_ld_wait();
+        float v[16];
 #pragma unroll
-        for (int I = 1; I < 4; ++I) {
-          const int i = 16 * I + lane;
-          float v[48];
-#pragma unroll
-          for (int c = 0; c < 16 * I; ++c)
-            v[c] = __uint_as_float(I == 1 ? r1[c] : (I == 2 ? r2[c] : (c < 32 ? r3a[c] : r3b[c - 32])));
-          if (warp == 0) {
-            const float bi = sBeta[i];
-#pragma unroll
-            for (int c = 0; c < 16 * I; c += 4)
-              *reinterpret_cast<uint2*>(sAh + i * LDH + c) = make_uint2(pack_f16(bi * v[c], bi * v[c + 1]), pack_f16(bi * v[c + 2], bi * v[c + 3]));
-          } else {
-#pragma unroll
-            for (int ch = 0; ch < 2 * I; ++ch) {
-              const float t8[8] = {v[ch * 8], v[ch * 8 + 1], v[ch * 8 + 2], v[ch * 8 + 3],
-                                   v[ch * 8 + 4], v[ch * 8 + 5], v[ch * 8 + 6], v[ch * 8 + 7]};
-              *reinterpret_cast<uint4*>(sm + OFF_P + sw128_offset(i, ch)) = pack8(t8);
-            }
-          }
+        for (int c = 0; c < 16; ++c) {
+          const int jj = 16 * cb + c;
+          const bool keep = isq ? jj <= i : jj < i;      // only the diagonal piece (cb == I) has entries to drop
+          v[c] = keep ? __uint_as_float(r[c]) * (isq ? 1.f : bi) : 0.f;
+        }
+        if (!isq) {
+          uint4* d = reinterpret_cast<uint4*>(sAh + i * LDH + 16 * cb);
+          d[0] = make_uint4(pack_f16(v[0], v[1]), pack_f16(v[2], v[3]), pack_f16(v[4], v[5]), pack_f16(v[6], v[7]));
+          d[1] = make_uint4(pack_f16(v[8], v[9]), pack_f16(v[10], v[11]), pack_f16(v[12], v[13]), pack_f16(v[14], v[15]));
+        } else {
+          *reinterpret_cast<uint4*>(sm + OFF_P + sw128_offset(i, 2 * cb)) = pack8(*reinterpret_cast<const float(*)[8]>(v));
+          *reinterpret_cast<uint4*>(sm + OFF_P + sw128_offset(i, 2 * cb + 1)) = pack8(*reinterpret_cast<const float(*)[8]>(v + 8));
         }
       }
     }
-    __syncthreads();                                     // everyone is done with the raw K and Q tiles
+    gsync();
+    // diagonal blocks where the clamp was hit: element by element, 136 pairs (j <= i) per block
+    for (int blk = 0; blk < 4; ++blk) {
+      if (!sFall[blk]) continue;
+      for (int qq = tid; qq < 136; qq += kPrepThreads) {
+        int il = 0;
+        while ((il + 1) * (il + 2) / 2 <= qq) ++il;
+        const int jl = qq - il * (il + 1) / 2;
+        const int i = blk * 16 + il, jj = blk * 16 + jl;
+        float kk = 0.f, qk = 0.f;
+#pragma unroll 2
+        for (int cc = 0; cc < 16; ++cc) {
+          const uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
+          float kif[8], qif[8], kjf[8], gi[8], gj[8];
+          unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(i, cc & 7)), kif);
+          unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + sw128_offset(i, cc & 7)), qif);
+          unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(jj, cc & 7)), kjf);
+          *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
+          *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
+          *reinterpret_cast<float4*>(gj) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8);
+          *reinterpret_cast<float4*>(gj + 4) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8 + 4);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float t = kjf[e] * ex2(gi[e] - gj[e]);
+            kk = fmaf(kif[e], t, kk);
+            qk = fmaf(qif[e], t, qk);
+          }
+        }
+        if (jj < i) sAh[i * LDH + jj] = __float2half_rn(sBeta[i] * kk);
+        *reinterpret_cast<__nv_bfloat16*>(sm + OFF_P + sw128_offset(i, jj >> 3) + (jj & 7) * 2) = __float2bfloat16_rn(qk);
+      }
+    }
+    gsync();                                     // everyone is done with the raw K and Q tiles
 
     // ---- operands rescaled in place: K <- K 2^G (for W), Q <- Q 2^G (for Q~); K e^{G_L - G} for the chain
     {
@@ -559,7 +601,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);  // one warp polls; the others sleep at the barrier
     mph ^= 1;
-    __syncthreads();                                     // (also makes sEG / sBE visible to everyone)
+    gsync();                                     // (also makes sEG / sBE visible to everyone)
     PP(4);
     tc_fence_after_sync();
     {
@@ -591,7 +633,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
   }
-  __syncthreads();
+  gsync();
   PP(5);
 
   // ---- op #3 Solve: T = (I + A)^-1
@@ -616,7 +658,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       sD[blk * 256 + q * 16 + c] = __float2half_rn(y[q]);
     }
   }
-  __syncthreads();
+  gsync();
   PP(6);
   {
     // the diagonal inverses go back in place (for level 2 and the final read) ...
@@ -632,17 +674,17 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       merge_store<2>(c2, sAh + hi * LDH + lo, LDH, 0, 0, lane);
     }
   }
-  __syncthreads();
+  gsync();
   PP(7);
   {
     // level 2: the 32x32 block (rows 32..63, columns 0..31); warp -> (16 columns, 8 rows) of the result
     const int mt = warp & 1, n2 = warp >> 1;
     float c2[1][4];
     merge_compute<32, 1>(c2, sAh, LDH, sAh + 32 * LDH, LDH, sAh + 32 * LDH + 32, LDH, mt, n2, lane);
-    __syncthreads();                                     // every warp has read A_10 before it is overwritten
+    gsync();                                     // every warp has read A_10 before it is overwritten
     merge_store<1>(c2, sAh + 32 * LDH, LDH, mt, n2, lane);
   }
-  __syncthreads();
+  gsync();
   PP(8);
 
   // ---- column-scaled copies of T as bf16 operand tiles: T^W = T diag(beta e^G), T^U = T diag(beta).
@@ -651,7 +693,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int i = tid >> 2, q4 = tid & 3;                // row, quarter (16 columns = two 16-byte pieces)
     const uint4 traw0 = *reinterpret_cast<const uint4*>(sAh + i * LDH + q4 * 16);
     const uint4 traw1 = *reinterpret_cast<const uint4*>(sAh + i * LDH + q4 * 16 + 8);
-    __syncthreads();
+    gsync();
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
       const int ch = q4 * 2 + q;
@@ -670,7 +712,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
   fence_proxy_async_smem();
   tc_fence_before_sync();
-  __syncthreads();
+  gsync();
   PP(9);
 
   // ---- op #4 W/U: W^T = K^T (T^W)^T, U^T = V^T (T^U)^T  (A operands feature-major straight from the TMA tiles)
@@ -691,7 +733,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
   if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
   mph ^= 1;
-  __syncthreads();
+  gsync();
   PP(10);
   tc_fence_after_sync();
   {
@@ -716,7 +758,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
   fence_proxy_async_smem();
   tc_fence_before_sync();
-  __syncthreads();
+  gsync();
   PP(11);
 
   // ---- chunk-local halves of op #6: (P W)^T = W^T P^T, O_loc^T = U^T P^T; the W and U images leave meanwhile
@@ -758,12 +800,12 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
   if (tid == 0) bulk_wait_read_1();                      // the W image was read; it receives the Q~ image
   mph ^= 1;
-  __syncthreads();
+  gsync();
   PP(12);
   tc_fence_after_sync();
   // Every MMA of this item is done, so the K / Q tile regions are free: start the next item's loads now
   // (its V tiles follow at the top of the loop, once the O_loc image has left their room).
-  const long long nxt = cjl + gridDim.x;
+  const long long nxt = cjl + vstride;
   if (tid == 0) {                                        // one thread works out where the next item is
     int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
     bool hn = nxt < p.total;
@@ -781,7 +823,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (tid == 0) bulk_wait_read_all();                  // the U image was read too
     fence_proxy_async_smem();
     tc_fence_before_sync();
-    __syncthreads();
+    gsync();
     if (tid == 0) {
       bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_WT, kImgBytes);
       bulk_commit();
@@ -793,7 +835,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // The accumulators were read: the next item's first MMA may overwrite them after this barrier.
   fence_proxy_async_smem();
   tc_fence_before_sync();
-  __syncthreads();
+  gsync();
   if (tid == 0) {
     bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
     bulk_commit();
@@ -806,8 +848,6 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   cjl = nxt; have = have_n; j = jn; jq = jqn; L = Ln; tok0 = tok0n;
   }  // work items
 
-  __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, 128);
   if (tid == 0) {
     if (*abort_flag) report_status(p.status, HA_LA_ERR_TIMEOUT);
     if (prev_cj >= 0) {
@@ -816,19 +856,24 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         fence_proxy_async_all();
         __threadfence();
         st_release_gpu(p.ws.flags + prev_cj, p.epoch);
+        if (prev_cj % p.HV == 0) HA_PROF_GT(prep, 512 + (int)(prev_cj / p.HV));
       } else {
         bulk_wait_read_all();                            // shared memory must outlive the bulk stores' reads
       }
     }
   }
+  tc_fence_before_sync();
+  __syncthreads();                                       // all groups are done with tensor memory
+  if (threadIdx.x < 32) tmem_dealloc(tmem_cta, G == 1 ? 256 : 512);
   HA_PROF(prep, 14);
+  if (threadIdx.x == 0) HA_PROF_GT(prep, 901);   // last writer wins: roughly the end of the kernel
 }
 
 }  // namespace
 
 template <bool KDA>
 static cudaError_t configure_prep_variant() {
-  const int smem = KDA ? kPrepSmemKda : kPrepSmem;
+  const int smem = KDA ? kPrepSmemKda : kGroups<KDA> * kGroupSmem;
   cudaError_t e = cudaFuncSetAttribute(tc_prep_kernel<KDA>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   // Same carve-out preference as the chain kernel: kernels that prefer different L1 / shared splits do not
@@ -840,9 +885,9 @@ static cudaError_t configure_prep_variant() {
 template <bool KDA>
 static cudaError_t launch_prep_variant(const PrepParams& pp, const CUtensorMap& mq, const CUtensorMap& mk,
                                        const CUtensorMap& mv, long long grid, cudaStream_t stream) {
-  const int smem = KDA ? kPrepSmemKda : kPrepSmem;
+  const int smem = KDA ? kPrepSmemKda : kGroups<KDA> * kGroupSmem;
   timer_mark(stream, "tc_prep");
-  tc_prep_kernel<KDA><<<(unsigned)grid, kPrepThreads, smem, stream>>>(mq, mk, mv, pp);
+  tc_prep_kernel<KDA><<<(unsigned)grid, kPrepThreads * kGroups<KDA>, smem, stream>>>(mq, mk, mv, pp);
   return cudaGetLastError();
 }
 
@@ -865,10 +910,12 @@ cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanVi
   if (pp.total == 0) return cudaSuccess;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  // resident CTAs; in the concurrent mode the SMs that hold a chain CTA are left out
-  long long slots = (long long)(sms - reserved_sms) * (p.variant == HA_LA_KDA ? 1 : 3);
-  if (slots < 1) slots = 1;
-  const long long grid = pp.total < slots ? pp.total : slots;
+  // one CTA per SM; in the concurrent mode the SMs that will hold a chain CTA are left out
+  const int groups = p.variant == HA_LA_KDA ? 1 : 3;
+  long long ctas = sms - reserved_sms;
+  if (ctas < 1) ctas = 1;
+  const long long need = (pp.total + groups - 1) / groups;
+  const long long grid = need < ctas ? need : ctas;
   return p.variant == HA_LA_KDA ? launch_prep_variant<true>(pp, mq, mk, mv, grid, stream)
                                 : launch_prep_variant<false>(pp, mq, mk, mv, grid, stream);
 }

@@ -63,6 +63,19 @@ def test_kda_slow_decay():
     helpers.check_parity(synth.make_inputs(w, seed=10))
 
 
+def test_kda_extreme_decay_inside_a_block():
+    """A few tokens forget almost everything in some channels (log-gate -90: a factor 2^-130).  Inside their
+    16-token block the tensor-core factorisation of the decay would need 2^+130, so the kernel has to take
+    its element-wise evaluation for those diagonal blocks; everything else stays on the tensor cores."""
+    w = synth.shrink(W["kda_8k"], seq_lens=[300], hk=1, hv=2)
+    inp = synth.make_inputs(w, seed=12)
+    g = inp["g"]
+    assert g.ndim == 3 and g.shape[-1] == 128
+    for tok in (5, 37, 70, 71, 200):
+        g[tok, :, ::7] = -90.0
+    helpers.check_parity(inp)
+
+
 def test_varlen_small_with_empty_and_tiny_sequences():
     w = synth.shrink(W["gdn_varlen"], seq_lens=[70, 0, 129, 64, 5, 1, 600], hk=2, hv=2)
     inp = synth.make_inputs(w, seed=13)
@@ -158,14 +171,21 @@ def test_tc_every_slice_width(nv, monkeypatch):
     helpers.check_parity(inp)
 
 
-def test_concurrent_prep_and_chain_mode(monkeypatch):
-    """Opt-in mode: the chain kernel runs next to the persistent prep kernel and takes each chunk as soon
-    as its flag is published.  Same results as the sequential mode, bit for bit."""
-    w = synth.shrink(W["gdn_layer_4k"], seq_lens=[2048], hk=4, hv=4)
+@pytest.mark.parametrize("case", ["gdn", "kda", "varlen"])
+def test_concurrent_prep_and_chain_mode(case, monkeypatch):
+    """Default mode when the chain CTAs need at most half of the SMs: the chain kernel runs next to the
+    persistent prep kernel and takes each chunk as soon as its flag is published.  HA_LA_TC_OVERLAP=0
+    forces the sequential mode.  Same results in both, bit for bit, call after call."""
+    if case == "gdn":
+        w = synth.shrink(W["gdn_layer_4k"], seq_lens=[2048], hk=4, hv=4)
+    elif case == "kda":
+        w = synth.shrink(W["kda_8k"], seq_lens=[1000], hk=2, hv=4)
+    else:
+        w = synth.shrink(W["gdn_varlen"], seq_lens=[700, 0, 65, 1500], hk=2, hv=2)
     inp = synth.make_inputs(w, seed=37)
     monkeypatch.setenv("HA_LA_TC_OVERLAP", "0")
     o_seq, h_seq, st_seq = helpers.run_gpu(inp)
-    monkeypatch.setenv("HA_LA_TC_OVERLAP", "1")
+    monkeypatch.delenv("HA_LA_TC_OVERLAP")
     o_con, h_con, st_con = helpers.run_gpu(inp)
     o_con2, h_con2, _ = helpers.run_gpu(inp)
     assert st_seq == 0 and st_con == 0
