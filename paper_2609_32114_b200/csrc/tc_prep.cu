@@ -237,6 +237,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   uint64_t* bar_load = reinterpret_cast<uint64_t*>(sm + OFF_BAR);
   uint64_t* bar_mma = bar_load + 1;
   uint64_t* bar_v = bar_load + 2;                        // the V tiles arrive on their own barrier
+  uint64_t* bar_g = bar_load + 7;                        // KDA: the log-gate rows of the next item
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_load + 3);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* sNext = reinterpret_cast<int*>(tmem_slot + 2);    // next item: have, j, jq, L, tok0 (written by thread 0)
@@ -255,6 +256,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     mbar_init(bar_load, 1);
     mbar_init(bar_mma, 1);
     mbar_init(bar_v, 1);
+    mbar_init(bar_g, 1);
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
@@ -320,19 +322,28 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   int j = 0, jq = 0, L = 0, tok0 = 0;
   bool have = cjl < p.total;
   if (have) { item_geom(cjl, j, jq, L, tok0); have = L > 0; }   // unused chunk slots come last
-  // GDN: warp 1 stages the log-gates and betas of an item in shared memory with cp.async (two tokens per lane),
-  // one item ahead, and scans them at the top of that item.
+  // Warp 1 stages the per-token scalars of an item one item ahead: GDN, log-gate and beta with cp.async (two
+  // tokens per lane), scanned at the top of that item; KDA, beta likewise and the 64 x 128 log-gate rows by
+  // bulk copies straight into the gate matrix (512 contiguous bytes per token).
   auto stage_gates = [&](int j_, int L_, int tok0_) {
-    if (!KDA && warp == 1) {
+    if (warp == 1) {
+      if (KDA && lane == 0) mbar_expect_tx(bar_g, (uint32_t)L_ * 512u);
+      __syncwarp();
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int t = lane + 32 * h;
         if (t < L_) {
-          cp_async4(sRaw + t, p.g + (size_t)(tok0_ + t) * p.HV + j_);
+          if (!KDA) cp_async4(sRaw + t, p.g + (size_t)(tok0_ + t) * p.HV + j_);
           cp_async4(sRaw + 64 + t, p.beta + (size_t)(tok0_ + t) * p.HV + j_);
+          if (KDA)
+            bulk_load(sm + OFF_G + t * LDG * 4, p.g + ((size_t)(tok0_ + t) * p.HV + j_) * 128, 512, bar_g);
         } else {
           sRaw[t] = 0.f;
           sRaw[64 + t] = 0.f;
+          if (KDA) {
+            float4* row = reinterpret_cast<float4*>(sm + OFF_G + t * LDG * 4);
+            for (int c = 0; c < 32; ++c) row[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
         }
       }
     }
@@ -352,27 +363,32 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     gsync();
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
     float* sGc = reinterpret_cast<float*>(sm + OFF_G);
+    PP(2);
     {
-      const float* gsrc = p.g + ((size_t)tok0 * p.HV + j) * 128;
-      for (int idx = tid; idx < 64 * 128; idx += kPrepThreads) {
-        const int i = idx >> 7, c = idx & 127;
-        sGc[i * LDG + c] = i < L ? gsrc[(size_t)i * p.HV * 128 + c] * 1.4426950408889634f : 0.f;
-      }
-      if (tid < 64) {
-        const float b = tid < L ? p.beta[(size_t)(tok0 + tid) * p.HV + j] : 0.f;
-        sBeta[tid] = b;
-        sBE[tid] = b;                                    // the gate factor lives in the K operand, not in T^W
-        sEG[tid] = 1.f;                                  // and Q is rescaled in place: E = identity
+      if (warp == 1) {
+        cp_async_wait_all();
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float b = sRaw[64 + lane + 32 * h];
+          sBeta[lane + 32 * h] = b;
+          sBE[lane + 32 * h] = b;                        // the gate factor lives in the K operand, not in T^W
+          sEG[lane + 32 * h] = 1.f;                      // and Q is rescaled in place: E = identity
+        }
       }
       // A and P start as zero (entries above the diagonal are never written)
       for (int idx = tid; idx < 64 * LDH * 2 / 16; idx += kPrepThreads) reinterpret_cast<uint4*>(sAh)[idx] = make_uint4(0, 0, 0, 0);
       for (int idx = tid; idx < 512; idx += kPrepThreads) reinterpret_cast<uint4*>(sm + OFF_P)[idx] = make_uint4(0, 0, 0, 0);
     }
+    if (warp == 0) mbar_wait(bar_g, lph, abort_flag);    // the raw log-gate rows (staged during the previous item)
     gsync();
+    PP(3);
     {
       const int c = tid & 127, r0 = (tid >> 7) * 32;     // two threads per channel, 32 rows each
       float acc = 0.f;
-      for (int i = 0; i < 32; ++i) { acc += sGc[(r0 + i) * LDG + c]; sGc[(r0 + i) * LDG + c] = acc; }
+      for (int i = 0; i < 32; ++i) {
+        acc = fmaf(sGc[(r0 + i) * LDG + c], 1.4426950408889634f, acc);
+        sGc[(r0 + i) * LDG + c] = acc;
+      }
     }
     gsync();
     if (tid >= 128) {
@@ -447,6 +463,39 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     fence_proxy_async_smem();
     tc_fence_before_sync();
     gsync();
+    // ---- operands rescaled in place: K <- K 2^G (for W), Q <- Q 2^G (for Q~); K e^{G_L - G} for the chain.
+    // The tensor cores read the K+ / Q+ / K- copies, not these tiles, so this runs while they work -- unless a
+    // diagonal block has to be evaluated again from the raw tiles first.
+    auto rescale_pass = [&]() {
+    {
+      const int i = tid >> 2;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int cc = (tid & 3) * 4 + q;
+        uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
+        const uint32_t off = sw128_offset(i, cc & 7);
+        float kf[8], qf[8], gi[8], gl[8], kd[8];
+        unpack8(*reinterpret_cast<const uint4*>(kt + off), kf);
+        unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + off), qf);
+        *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
+        *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
+        *reinterpret_cast<float4*>(gl) = *reinterpret_cast<const float4*>(sGc + 63 * LDG + cc * 8);
+        *reinterpret_cast<float4*>(gl + 4) = *reinterpret_cast<const float4*>(sGc + 63 * LDG + cc * 8 + 4);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float eg = ex2(gi[e]);
+          kd[e] = kf[e] * ex2(gl[e] - gi[e]);
+          kf[e] *= eg;
+          qf[e] *= eg;
+        }
+        *reinterpret_cast<uint4*>(kt + off) = pack8(kf);
+        *reinterpret_cast<uint4*>(kt + 8192 + off) = pack8(qf);
+        *reinterpret_cast<uint4*>(sm + OFF_KD + (cc >> 3) * 8192 + off) = pack8(kd);
+      }
+    }
+    };
+    PP(0);
+    const bool anyfall = (sFall[0] | sFall[1] | sFall[2] | sFall[3]) != 0;
     if (tid == 0) {                        // block-row I: D_I[128 x 16 (I + 1)] = [all K+ / Q+ rows] (K-^(I))^T;
       tc_fence_after_sync();               // only rows 32 I .. 32 I + 31 (K+_I, Q+_I) of D_I are used
 #pragma unroll
@@ -464,9 +513,11 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       umma_commit(bar_mma);
       publish_prev();
     }
+    if (!anyfall) rescale_pass();
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
     mph ^= 1;
     gsync();
+    PP(1);
     tc_fence_after_sync();
     {
       // Block-row I sits in tensor-memory lanes 32 I .. 32 I + 31: lanes 0..15 the K+ rows (-> A), 16..31 the Q+
@@ -498,67 +549,43 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
     }
-    gsync();
-    // diagonal blocks where the clamp was hit: element by element, 136 pairs (j <= i) per block
-    for (int blk = 0; blk < 4; ++blk) {
-      if (!sFall[blk]) continue;
-      for (int qq = tid; qq < 136; qq += kPrepThreads) {
-        int il = 0;
-        while ((il + 1) * (il + 2) / 2 <= qq) ++il;
-        const int jl = qq - il * (il + 1) / 2;
-        const int i = blk * 16 + il, jj = blk * 16 + jl;
-        float kk = 0.f, qk = 0.f;
-#pragma unroll 2
-        for (int cc = 0; cc < 16; ++cc) {
-          const uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
-          float kif[8], qif[8], kjf[8], gi[8], gj[8];
-          unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(i, cc & 7)), kif);
-          unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + sw128_offset(i, cc & 7)), qif);
-          unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(jj, cc & 7)), kjf);
-          *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
-          *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
-          *reinterpret_cast<float4*>(gj) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8);
-          *reinterpret_cast<float4*>(gj + 4) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8 + 4);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const float t = kjf[e] * ex2(gi[e] - gj[e]);
-            kk = fmaf(kif[e], t, kk);
-            qk = fmaf(qif[e], t, qk);
+    if (anyfall) {
+      gsync();
+      // diagonal blocks where the clamp was hit: element by element, 136 pairs (j <= i) per block
+      for (int blk = 0; blk < 4; ++blk) {
+        if (!sFall[blk]) continue;
+        for (int qq = tid; qq < 136; qq += kPrepThreads) {
+          int il = 0;
+          while ((il + 1) * (il + 2) / 2 <= qq) ++il;
+          const int jl = qq - il * (il + 1) / 2;
+          const int i = blk * 16 + il, jj = blk * 16 + jl;
+          float kk = 0.f, qk = 0.f;
+  #pragma unroll 2
+          for (int cc = 0; cc < 16; ++cc) {
+            const uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
+            float kif[8], qif[8], kjf[8], gi[8], gj[8];
+            unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(i, cc & 7)), kif);
+            unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + sw128_offset(i, cc & 7)), qif);
+            unpack8(*reinterpret_cast<const uint4*>(kt + sw128_offset(jj, cc & 7)), kjf);
+            *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
+            *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
+            *reinterpret_cast<float4*>(gj) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8);
+            *reinterpret_cast<float4*>(gj + 4) = *reinterpret_cast<const float4*>(sGc + jj * LDG + cc * 8 + 4);
+  #pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float t = kjf[e] * ex2(gi[e] - gj[e]);
+              kk = fmaf(kif[e], t, kk);
+              qk = fmaf(qif[e], t, qk);
+            }
           }
+          if (jj < i) sAh[i * LDH + jj] = __float2half_rn(sBeta[i] * kk);
+          *reinterpret_cast<__nv_bfloat16*>(sm + OFF_P + sw128_offset(i, jj >> 3) + (jj & 7) * 2) = __float2bfloat16_rn(qk);
         }
-        if (jj < i) sAh[i * LDH + jj] = __float2half_rn(sBeta[i] * kk);
-        *reinterpret_cast<__nv_bfloat16*>(sm + OFF_P + sw128_offset(i, jj >> 3) + (jj & 7) * 2) = __float2bfloat16_rn(qk);
       }
+      gsync();                                   // everyone is done with the raw K and Q tiles
+      rescale_pass();
     }
-    gsync();                                     // everyone is done with the raw K and Q tiles
 
-    // ---- operands rescaled in place: K <- K 2^G (for W), Q <- Q 2^G (for Q~); K e^{G_L - G} for the chain
-    {
-      const int i = tid >> 2;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int cc = (tid & 3) * 4 + q;
-        uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
-        const uint32_t off = sw128_offset(i, cc & 7);
-        float kf[8], qf[8], gi[8], gl[8], kd[8];
-        unpack8(*reinterpret_cast<const uint4*>(kt + off), kf);
-        unpack8(*reinterpret_cast<const uint4*>(kt + 8192 + off), qf);
-        *reinterpret_cast<float4*>(gi) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8);
-        *reinterpret_cast<float4*>(gi + 4) = *reinterpret_cast<const float4*>(sGc + i * LDG + cc * 8 + 4);
-        *reinterpret_cast<float4*>(gl) = *reinterpret_cast<const float4*>(sGc + 63 * LDG + cc * 8);
-        *reinterpret_cast<float4*>(gl + 4) = *reinterpret_cast<const float4*>(sGc + 63 * LDG + cc * 8 + 4);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float eg = ex2(gi[e]);
-          kd[e] = kf[e] * ex2(gl[e] - gi[e]);
-          kf[e] *= eg;
-          qf[e] *= eg;
-        }
-        *reinterpret_cast<uint4*>(kt + off) = pack8(kf);
-        *reinterpret_cast<uint4*>(kt + 8192 + off) = pack8(qf);
-        *reinterpret_cast<uint4*>(sm + OFF_KD + (cc >> 3) * 8192 + off) = pack8(kd);
-      }
-    }
   } else {
     // ---- op #1 Gate: inclusive scan of the log-gate over the chunk (warp 1, tokens lane and lane + 32)
     if (warp == 1) {
