@@ -68,27 +68,27 @@ int sm_count() {
   return n;
 }
 
-// Value channels per chain CTA: the narrowest slice that still gives every CTA its own SM.
-int pick_nv(const Problem& p) {
-  if (const char* e = getenv("HA_LA_TC_NV")) {
-    const int v = atoi(e);
-    if (v == 32 || v == 64 || v == 128) return v;
-  }
-  const long long chains = (long long)p.N * p.HV;
-  const int sms = sm_count();
-  if (chains * 4 <= sms) return 32;
-  if (chains * 2 <= sms) return 64;
-  return 128;
-}
-
 std::atomic<int32_t> g_epoch{0};
 
-bool want_concurrent(const Problem& p, int nv) {
-  if (g_timer) return false;                             // per-kernel timing wants one kernel at a time
-  const char* e = getenv("HA_LA_TC_OVERLAP");
-  if (e && e[0] == '0') return false;
-  const long long chain_ctas = (long long)p.N * p.HV * (128 / nv);
-  return chain_ctas * 2 <= sm_count() && p.max_chunks > 1;
+// Slice width (value channels per chain CTA) and launch mode.  The chain kernel is bound by the latency of its
+// two MMA round trips per chunk, which grows with the slice width (about 0.9 / 1.4 / 1.95 us per chunk at 32 /
+// 64 / 128 channels on B200) and does not depend on the number of CTAs: take the narrowest slice that still
+// gives every CTA an SM of its own.  Concurrent mode when those CTAs leave at least half of the SMs to the prep
+// kernel and the slice is the narrow one (with 64-channel slices the overlap measured no gain over running
+// the two kernels back to back with 32-channel slices).
+struct TcPlan { int nv; bool concurrent; };
+
+TcPlan plan_tc(const Problem& p) {
+  const int sms = sm_count();
+  const long long chains = (long long)p.N * p.HV;
+  int nv = chains * 4 <= sms ? 32 : (chains * 2 <= sms ? 64 : 128);
+  if (const char* e = getenv("HA_LA_TC_NV")) {
+    const int v = atoi(e);
+    if (v == 32 || v == 64 || v == 128) nv = v;
+  }
+  bool conc = !g_timer && p.max_chunks > 1 && nv == 32 && chains * 4 * 2 <= sms;   // (timing wants one kernel at a time)
+  if (const char* e = getenv("HA_LA_TC_OVERLAP")) conc = conc && e[0] != '0';
+  return TcPlan{nv, conc};
 }
 
 }  // namespace
@@ -109,9 +109,9 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
       !make_map(&mv, a.v, p.T_total, p.HV))
     return cudaErrorInvalidValue;
   const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
-  const int nv = pick_nv(p);
-
-  const bool concurrent = want_concurrent(p, nv);
+  const TcPlan tp = plan_tc(p);
+  const int nv = tp.nv;
+  const bool concurrent = tp.concurrent;
   // Configure (and load) both kernels before anything is enqueued: loading a kernel for the first time can
   // wait for the device, and in the concurrent mode the chain kernel would be spinning meanwhile.
   cudaError_t ce = configure_tc_prep(p);

@@ -304,8 +304,10 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
           if (c0 > 0) load_img32(stage + Cfg::OFF_U, i, cg0 + c0, pre);
 #pragma unroll
           for (int q = 0; q < 32; ++q) d[q] = (pre[q] - d[q]) * dec;
+          if (c0 == 0) HA_PROF(chain, 8 * c + 6);
           store_brow32<NV, 64>(sUt, i, cg0 + c0, d);
         }
+        HA_PROF(chain, 8 * c + 7);
         fence_proxy_async_smem();
         tc_fence_before_sync();
         named_arrive(BAR_U_READY, NCOMP / 2 + 32);

@@ -92,9 +92,6 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
 // 1-D bulk copy shared -> global (same alignment rules).  One thread issues, commits the group and,
 // before the shared buffer is reused or the CTA exits, waits until the group has been read.
 __device__ __forceinline__ void bulk_store(void* gdst, const void* ssrc, uint32_t bytes) {
-#ifdef HA_EXP_NOSTORE
-  return;
-#endif
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                ::"l"(reinterpret_cast<uint64_t>(gdst)), "r"(smem_u32(ssrc)), "r"(bytes) : "memory");
 }
