@@ -307,8 +307,8 @@ def main():
     kernel_alg_bytes = {"simt_prefill": alg_bytes, "tc_prep": in_bytes, "tc_chain": out_bytes, "plan": 0.0}
     # DRAM bytes per launch of that kernel from one ncu --set full capture of this workload
     # (profiles/tc_prep_chain_gdn_layer_4k_ncu_full.md, profiles/tc_prep_chain_kda_8k_ncu_full.md); cold-cache replays
-    ncu_traffic = {("gdn_layer_4k", "tc_chain"): 84.71e6 + 5.53e6, ("gdn_layer_4k", "tc_prep"): 50.92e6 + 17.64e6,
-                   ("kda_8k", "tc_prep"): 336.68e6 + 291.53e6, ("kda_8k", "tc_chain"): 338.72e6 + 56.35e6}
+    ncu_traffic = {("gdn_layer_4k", "tc_chain"): 84.71e6 + 5.63e6, ("gdn_layer_4k", "tc_prep"): 50.92e6 + 15.10e6,
+                   ("kda_8k", "tc_prep"): 336.68e6 + 290.63e6, ("kda_8k", "tc_chain"): 338.74e6 + 57.43e6}
     dom_bytes = kernel_alg_bytes.get(dom, alg_bytes)
     dom_s = kernel_ms[dom] / 1e3
     achieved = dom_bytes / dom_s / 1e9
@@ -318,7 +318,9 @@ def main():
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic.get((w.name, dom)),
                 "kernel_alg_bytes": dom_bytes, "peak_source": peaks["source"],
-                "kernel_ms": kernel_ms,
+                "kernel_ms": kernel_ms,      # each kernel alone (sequential launches with events in between)
+                "launch_mode": "sequential" if os.environ.get("HA_LA_TC_OVERLAP", "1")[:1] == "0" else
+                               "default (prep and chain kernels overlap when the chain leaves SMs free)",
                 "path": {"bound": "hbm" if t_hbm >= t_flop else "tensor", "roofline_us": 1e6 * max(t_hbm, t_flop),
                          "measured_us": 1e6 * path_s, "frac": max(t_hbm, t_flop) / path_s,
                          "achieved_gbs": alg_bytes / path_s / 1e9, "achieved_tflops": alg_flops / path_s / 1e12,

@@ -13,16 +13,17 @@
 #include <stdlib.h>
 
 #include <atomic>
+#include <random>
 
 #include "tc_common.cuh"
 
 namespace ha_la {
 
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int32_t epoch,
+                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int64_t epoch,
                            int reserved_sms, cudaStream_t stream);
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                            const CUtensorMap& mk, int nv, int32_t epoch, bool dependent, cudaStream_t stream);
+                            const CUtensorMap& mk, int nv, int64_t epoch, bool dependent, cudaStream_t stream);
 
 cudaError_t configure_tc_prep(const Problem& p);
 cudaError_t configure_tc_chain(const Problem& p, int nv);
@@ -68,7 +69,17 @@ int sm_count() {
   return n;
 }
 
-std::atomic<int32_t> g_epoch{0};
+std::atomic<uint32_t> g_calls{0};
+
+// Epoch of a concurrent-mode call: (random per-process tag, never 0) << 32 | call counter.
+int64_t next_epoch() {
+  static const uint32_t tag = [] {
+    std::random_device rd;
+    uint32_t t = rd();
+    return t ? t : 0x9e3779b9u;
+  }();
+  return (int64_t)(((uint64_t)tag << 32) | g_calls.fetch_add(1));
+}
 
 // Slice width (value channels per chain CTA) and launch mode.  The chain kernel is bound by the latency of its
 // two MMA round trips per chunk, which grows with the slice width (about 0.9 / 1.4 / 1.95 us per chunk at 32 /
@@ -118,11 +129,10 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   if (ce != cudaSuccess) return ce;
   ce = configure_tc_chain(p, nv);
   if (ce != cudaSuccess) return ce;
-  int32_t epoch = 0;                                     // 0 means "sequential"
+  int64_t epoch = 0;                                     // 0 means "sequential"
   int reserved_sms = 0;
   if (concurrent) {
-    epoch = g_epoch.fetch_add(1) + 1;
-    if (epoch == 0) epoch = g_epoch.fetch_add(1) + 1;
+    epoch = next_epoch();
     reserved_sms = p.N * p.HV * (128 / nv);              // a chain CTA fills its SM
   }
   cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, reserved_sms, stream);

@@ -66,7 +66,7 @@ struct ChainParams {
   TcWorkspace ws;
   int HK, HV;
   float scale;
-  int32_t epoch;               // != 0: the prep kernel runs concurrently; wait for ws.flags[cj] == epoch per chunk
+  int64_t epoch;               // != 0: the prep kernel runs concurrently; wait for ws.flags[cj] == epoch per chunk
                                // == 0: wait for the whole prep grid before the first workspace read
   int32_t* status;
 };
@@ -189,7 +189,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
           const int cc = c + lane;
           bool ok = false;
           if (cc < nchunks)
-            ok = *reinterpret_cast<const volatile int32_t*>(p.ws.flags + (size_t)(chunk0 + cc) * p.HV + j) == p.epoch;
+            ok = *reinterpret_cast<const volatile int64_t*>(p.ws.flags + (size_t)(chunk0 + cc) * p.HV + j) == p.epoch;
           const unsigned m = __ballot_sync(0xffffffffu, ok);
           got = __ffs(~m) - 1;                           // leading published chunks (32 when all are)
           if (got < 0) got = 32;
@@ -413,7 +413,7 @@ cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, int nv, in
 }  // namespace
 
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                            const CUtensorMap& mk, int nv, int32_t epoch, bool dependent, cudaStream_t stream) {
+                            const CUtensorMap& mk, int nv, int64_t epoch, bool dependent, cudaStream_t stream) {
   ChainParams cp;
   cp.h0 = a.h0; cp.hT = a.hT; cp.o = a.o;
   cp.seq_tok0 = plan.seq_tok0; cp.seq_len = plan.seq_len; cp.seq_chunk0 = plan.seq_chunk0;

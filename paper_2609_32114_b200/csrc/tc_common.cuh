@@ -5,8 +5,10 @@
 //   u   [cj] : 16 KiB  U image
 //   ol  [cj] : 16 KiB  O_loc image
 //   kd  [cj] : 16 KiB  KDA only: K e^{G_L - G}, in the shared-memory layout of the TMA K tile
-//   flg [cj] : int32   set to the call's epoch by the prep CTA once everything above is in memory; the
-//                      chain kernel, when it runs concurrently with the prep kernel, waits for it per chunk
+//   flg [cj] : int64   set to the call's epoch by the prep CTA once everything above is in memory; the
+//                      chain kernel, when it runs concurrently with the prep kernel, waits for it per chunk.
+//                      An epoch is a per-process random 32-bit tag and a call counter, so that whatever the
+//                      caller's workspace held before cannot pass for "published" (nothing is ever cleared)
 //   sc  [cj] : 192 floats  e^{G_L - G_i} for the 64 tokens, then e^{G_L} for the 128 key channels
 // An "image" is a 128 x 64 bf16 matrix stored feature-major: row r (key or value channel) holds the
 // 64 tokens of the chunk in 128 bytes, and the eight 16-byte pieces of a row are stored at piece
@@ -26,13 +28,13 @@ struct TcWorkspace {
   uint8_t* u;
   uint8_t* ol;
   uint8_t* kd;      // KDA only
-  int32_t* flags;
+  int64_t* flags;
   float* sc;
 };
 
 inline __host__ size_t tc_ws_bytes_for(size_t ncj, bool kda) {
   return ncj * (2 * kImgBytes + kImgBytes + kImgBytes + (kda ? kImgBytes : 0)) +
-         align_up(ncj * kScFloats * sizeof(float), 1024) + align_up(ncj * sizeof(int32_t), 1024);
+         align_up(ncj * kScFloats * sizeof(float), 1024) + align_up(ncj * sizeof(int64_t), 1024);
 }
 
 inline __host__ TcWorkspace tc_ws_view(void* base, size_t ncj, bool kda) {
@@ -43,7 +45,7 @@ inline __host__ TcWorkspace tc_ws_view(void* base, size_t ncj, bool kda) {
   w.ol = b;                      b += ncj * kImgBytes;
   w.kd = kda ? b : nullptr;      b += kda ? ncj * kImgBytes : 0;
   w.sc = reinterpret_cast<float*>(b);  b += align_up(ncj * kScFloats * sizeof(float), 1024);
-  w.flags = reinterpret_cast<int32_t*>(b);
+  w.flags = reinterpret_cast<int64_t*>(b);
   return w;
 }
 

@@ -87,7 +87,7 @@ struct PrepParams {
   TcWorkspace ws;
   int HK, HV;
   long long total;        // work items = chunk slots x V-heads
-  int32_t epoch;          // published to ws.flags[cj] when this CTA's results are in memory (0: do not publish)
+  int64_t epoch;          // published to ws.flags[cj] when this CTA's results are in memory (0: do not publish)
   int32_t* status;
 };
 
@@ -925,7 +925,7 @@ cudaError_t configure_tc_prep(const Problem& p) {
 }
 
 cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int32_t epoch,
+                           const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int64_t epoch,
                            int reserved_sms, cudaStream_t stream) {
   PrepParams pp;
   pp.epoch = epoch;

@@ -193,3 +193,32 @@ def test_concurrent_prep_and_chain_mode(case, monkeypatch):
     np.testing.assert_array_equal(h_con, h_seq)
     np.testing.assert_array_equal(o_con2, o_seq)
     helpers.check_parity(inp)
+
+
+def test_workspace_contents_do_not_matter():
+    """The workspace is scratch: whatever it holds on entry (small integers, all ones, an earlier call's
+    flags) must not change the result -- in particular not pass for a 'chunk is ready' flag."""
+    import torch
+    import paper_2609_32114_b200 as ha
+
+    w = synth.shrink(W["gdn_layer_4k"], seq_lens=[1500], hk=2, hv=4)
+    inp = synth.make_inputs(w, seed=41)
+    d = helpers.to_device(inp)
+
+    def call(ws=None):
+        o, hT, st, ws_out = ha.ha_la_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"], variant=w.variant, h0=d["h0"],
+                                             cu_seqlens=d["cu_seqlens"], max_seqlen=d["max_seqlen"], workspace=ws)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        return o.clone(), hT.clone(), ws_out
+
+    o0, h0, ws0 = call()
+    for fill in (0x01, 0xFF, 0x00):
+        ws = torch.full_like(ws0, fill)
+        o1, h1, _ = call(ws)
+        assert torch.equal(o1, o0) and torch.equal(h1, h0)
+    ints = torch.arange(ws0.numel() // 4, dtype=torch.int32, device=ws0.device) % 64   # small counters everywhere
+    o2, h2, _ = call(ints.view(torch.uint8))
+    assert torch.equal(o2, o0) and torch.equal(h2, h0)
+    o3, h3, _ = call(ws0)                                                                # an earlier call's workspace
+    assert torch.equal(o3, o0) and torch.equal(h3, h0)
