@@ -222,3 +222,41 @@ def test_workspace_contents_do_not_matter():
     assert torch.equal(o2, o0) and torch.equal(h2, h0)
     o3, h3, _ = call(ws0)                                                                # an earlier call's workspace
     assert torch.equal(o3, o0) and torch.equal(h3, h0)
+
+
+def test_back_to_back_calls_share_a_workspace():
+    """Many calls queued on one stream without synchronising in between, alternating between two problems
+    of different shape that share one workspace (so every call sees the other's leftovers and the
+    launch-mode switches between concurrent and sequential): results must equal the first call's."""
+    import torch
+    import paper_2609_32114_b200 as ha
+
+    wa = synth.shrink(W["gdn_layer_4k"], seq_lens=[1024], hk=2, hv=2)           # few chains: concurrent mode
+    wb = synth.shrink(W["gdn_varlen"], seq_lens=[200, 0, 333, 64] * 10, hk=2, hv=4)   # 160 chains: sequential
+    ia, ib = synth.make_inputs(wa, seed=43), synth.make_inputs(wb, seed=44)
+    da, db = helpers.to_device(ia), helpers.to_device(ib)
+
+    def call(d, w, ws):
+        return ha.ha_la_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"], variant=w.variant, h0=d["h0"],
+                                cu_seqlens=d["cu_seqlens"], max_seqlen=d["max_seqlen"], workspace=ws)
+
+    _, _, _, ws_a = call(da, wa, None)
+    _, _, _, ws_b = call(db, wb, None)
+    ws = ws_a if ws_a.numel() >= ws_b.numel() else ws_b
+    ref_a = call(da, wa, ws)
+    ref_b = call(db, wb, ws)
+    torch.cuda.synchronize()
+    ref_a = (ref_a[0].clone(), ref_a[1].clone())
+    ref_b = (ref_b[0].clone(), ref_b[1].clone())
+    outs = []
+    for it in range(12):
+        d, w = (da, wa) if it % 2 == 0 else (db, wb)
+        o, hT, st, _ = call(d, w, ws)
+        outs.append((o.clone(), hT.clone(), st))                 # clones are queued on the same stream, in order
+    torch.cuda.synchronize()
+    for it, (o, hT, st) in enumerate(outs):
+        ref = ref_a if it % 2 == 0 else ref_b
+        assert int(st.item()) == 0
+        assert torch.equal(o, ref[0]) and torch.equal(hT, ref[1]), f"call {it} differs"
+    helpers.check_parity(ia)
+    helpers.check_parity(ib)
