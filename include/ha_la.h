@@ -77,7 +77,7 @@ typedef struct {
   const void*  q;         /* [B, T, HK, d_k] contiguous, token-major                         */
   const void*  k;         /* [B, T, HK, d_k]                                                 */
   const void*  v;         /* [B, T, HV, d_v]                                                 */
-  const float* g;         /* GDN [B, T, HV]; KDA [B, T, HV, d_k]; log-gate                   */
+  const float* g;         /* GDN [B, T, HV]; KDA [B, T, HV, d_k] (16-byte aligned); log-gate */
   const float* beta;      /* [B, T, HV]                                                      */
   const float* h0;        /* [N, HV, d_k, d_v] fp32 or NULL (zeros); N = B or num_seqs       */
   const int32_t* cu_seqlens; /* device int32 [num_seqs+1], cu[0]=0, non-decreasing,

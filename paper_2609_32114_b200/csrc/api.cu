@@ -108,6 +108,7 @@ int ha_la_prefill(const ha_la_prefill_args* a, void* cuda_stream) {
   if (al16 & 15) return HA_LA_ERR_INVALID_ARG;
   if (((uintptr_t)a->g | (uintptr_t)a->beta | (uintptr_t)a->cu_seqlens | (uintptr_t)a->status_word) & 3)
     return HA_LA_ERR_INVALID_ARG;
+  if (a->variant == HA_LA_KDA && ((uintptr_t)a->g & 15)) return HA_LA_ERR_INVALID_ARG;   // fetched by bulk copies
 
   size_t need = 0;
   rc = ha_la_prefill_workspace_bytes(a, &need);

@@ -37,7 +37,8 @@ HA_PROF_DECL(prep)
 
 namespace {
 
-constexpr int kPrepThreads = 256;        // threads of one work group (a CTA holds kGroups of them)
+constexpr int kPrepThreads = 256;        // threads of one work group that run every phase (a CTA holds kGroups groups)
+constexpr int kKdaThreads = 512;         // KDA: the group has 8 more warps, which only run the gate-dependent passes
 constexpr int LDH = 72;                  // row stride (halfs) of the fp16 64x64 matrix A / T
 
 // shared-memory map (bytes from the 1024-aligned base); 73.3 KiB, so that three CTAs fit one SM
@@ -74,7 +75,8 @@ constexpr uint32_t KQP_KB = 128 * 128;
 constexpr uint32_t OFF_KM = OFF_KQP + 2 * KQP_KB;         // [kb][160 rows][128 B], K-major, swizzled
 constexpr uint32_t KM_KB = 160 * 128;
 constexpr uint32_t OFF_FALL = OFF_KM + 2 * KM_KB;         // int[4]: diagonal block needs the element-wise evaluation
-constexpr uint32_t kPrepSmemKda = OFF_FALL + 16;
+constexpr uint32_t OFF_QT = OFF_FALL + 16;                // float[4][128]: per-channel totals of the scan's four quarters
+constexpr uint32_t kPrepSmemKda = OFF_QT + 4 * 128 * 4;
 constexpr float kMaxUpExp = 100.f;                        // largest exponent (base 2) allowed in a K- factor
 static_assert(kPrepSmemKda <= 227 * 1024, "KDA shared memory budget");
 
@@ -216,16 +218,19 @@ __device__ __forceinline__ void store_half_row(const float (&v)[32], int row, in
 }
 
 template <bool KDA>
-__global__ void __launch_bounds__(kPrepThreads * kGroups<KDA>, 1)
+__global__ void __launch_bounds__(KDA ? kKdaThreads : kPrepThreads * kGroups<KDA>, 1)
 tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, PrepParams p) {
   constexpr int G = kGroups<KDA>;
   extern __shared__ __align__(1024) uint8_t smem_raw[];  // no static shared memory in this kernel: 1024-aligned
-  const int grp = threadIdx.x / kPrepThreads;            // work group of this thread
+  constexpr int NT = KDA ? kKdaThreads : kPrepThreads;   // threads of a work group
+  const int grp = threadIdx.x / NT;                      // work group of this thread
   uint8_t* sm = smem_raw + grp * kGroupSmem;
-  auto gsync = [&]() {                                   // barrier of one work group
-    if (G == 1) __syncthreads();
-    else asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "r"(kPrepThreads) : "memory");
+  auto gsync = [&]() {                                   // barrier of the 8 warps of a group that run every phase
+    asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "r"(kPrepThreads) : "memory");
+  };
+  auto bsync = [&]() {                                   // KDA: barrier of all 16 warps of the group
+    asm volatile("bar.sync 8, %0;" ::"r"(kKdaThreads) : "memory");
   };
   __half* sAh = reinterpret_cast<__half*>(sm + OFF_A);  // A, then T in place
   __half* sD = reinterpret_cast<__half*>(sm + OFF_D);
@@ -242,8 +247,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* sNext = reinterpret_cast<int*>(tmem_slot + 2);    // next item: have, j, jq, L, tok0 (written by thread 0)
 
-  const int tid = threadIdx.x % kPrepThreads;
+  const int tid = threadIdx.x % NT;
   const int warp = tid >> 5, lane = tid & 31;
+  const bool is_main = !KDA || tid < kPrepThreads;       // KDA: warps 8..15 only help with the gate-dependent passes
   if (smem_u32(smem_raw) & 1023u) {                            // the swizzled layouts need it; never seen to fail
     if (threadIdx.x == 0) report_status(p.status, HA_LA_ERR_DEVICE_CHECK);
     return;
@@ -327,23 +333,29 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // bulk copies straight into the gate matrix (512 contiguous bytes per token).
   auto stage_gates = [&](int j_, int L_, int tok0_) {
     if (warp == 1) {
-      if (KDA && lane == 0) mbar_expect_tx(bar_g, (uint32_t)L_ * 512u);
-      __syncwarp();
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int t = lane + 32 * h;
         if (t < L_) {
           if (!KDA) cp_async4(sRaw + t, p.g + (size_t)(tok0_ + t) * p.HV + j_);
           cp_async4(sRaw + 64 + t, p.beta + (size_t)(tok0_ + t) * p.HV + j_);
-          if (KDA)
-            bulk_load(sm + OFF_G + t * LDG * 4, p.g + ((size_t)(tok0_ + t) * p.HV + j_) * 128, 512, bar_g);
         } else {
           sRaw[t] = 0.f;
           sRaw[64 + t] = 0.f;
-          if (KDA) {
-            float4* row = reinterpret_cast<float4*>(sm + OFF_G + t * LDG * 4);
-            for (int c = 0; c < 32; ++c) row[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-          }
+        }
+      }
+    }
+    if (KDA && warp == 8) {                              // a helper warp: off the other warps' critical path
+      if (lane == 0) mbar_expect_tx(bar_g, (uint32_t)L_ * 512u);
+      __syncwarp();
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int t = lane + 32 * h;
+        if (t < L_) {
+          bulk_load(sm + OFF_G + t * LDG * 4, p.g + ((size_t)(tok0_ + t) * p.HV + j_) * 128, 512, bar_g);
+        } else {
+          float4* row = reinterpret_cast<float4*>(sm + OFF_G + t * LDG * 4);
+          for (int c = 0; c < 32; ++c) row[c] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
       }
     }
@@ -360,9 +372,11 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (prev_cj >= 0) bulk_wait_read_all();
       issue_v(j, tok0);
     }
-    gsync();
+    bsync();
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
     float* sGc = reinterpret_cast<float*>(sm + OFF_G);
+    float* sQt = reinterpret_cast<float*>(sm + OFF_QT);    // totals of the four 16-row quarters of the scan
+    int* sFall = reinterpret_cast<int*>(sm + OFF_FALL);
     PP(2);
     {
       if (warp == 1) {
@@ -375,29 +389,32 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           sEG[lane + 32 * h] = 1.f;                      // and Q is rescaled in place: E = identity
         }
       }
+      if (tid < 4) sFall[tid] = 0;
       // A and P start as zero (entries above the diagonal are never written)
-      for (int idx = tid; idx < 64 * LDH * 2 / 16; idx += kPrepThreads) reinterpret_cast<uint4*>(sAh)[idx] = make_uint4(0, 0, 0, 0);
-      for (int idx = tid; idx < 512; idx += kPrepThreads) reinterpret_cast<uint4*>(sm + OFF_P)[idx] = make_uint4(0, 0, 0, 0);
+      for (int idx = tid; idx < 64 * LDH * 2 / 16; idx += NT) reinterpret_cast<uint4*>(sAh)[idx] = make_uint4(0, 0, 0, 0);
+      for (int idx = tid; idx < 512; idx += NT) reinterpret_cast<uint4*>(sm + OFF_P)[idx] = make_uint4(0, 0, 0, 0);
     }
     if (warp == 0) mbar_wait(bar_g, lph, abort_flag);    // the raw log-gate rows (staged during the previous item)
-    gsync();
+    bsync();
     PP(3);
+    const int sc_c = tid & 127, sc_q = tid >> 7;         // scan: four threads per channel, 16 rows each
     {
-      const int c = tid & 127, r0 = (tid >> 7) * 32;     // two threads per channel, 32 rows each
       float acc = 0.f;
-      for (int i = 0; i < 32; ++i) {
-        acc = fmaf(sGc[(r0 + i) * LDG + c], 1.4426950408889634f, acc);
-        sGc[(r0 + i) * LDG + c] = acc;
+      for (int i = 0; i < 16; ++i) {
+        acc = fmaf(sGc[(16 * sc_q + i) * LDG + sc_c], 1.4426950408889634f, acc);
+        sGc[(16 * sc_q + i) * LDG + sc_c] = acc;
       }
+      sQt[sc_q * 128 + sc_c] = acc;
     }
-    gsync();
-    if (tid >= 128) {
-      const int c = tid & 127;
-      const float add = sGc[31 * LDG + c];
-      for (int i = 32; i < 64; ++i) sGc[i * LDG + c] += add;
+    bsync();
+    if (sc_q > 0) {
+      float add = sQt[sc_c];
+      if (sc_q > 1) add += sQt[128 + sc_c];
+      if (sc_q > 2) add += sQt[256 + sc_c];
+      for (int i = 0; i < 16; ++i) sGc[(16 * sc_q + i) * LDG + sc_c] += add;
     }
     mbar_wait(bar_load, lph, abort_flag);                // every thread reads the K / Q tiles below
-    gsync();
+    bsync();
     PP(4);
 
     // ---- op #2 KKT and the masked Q K^T with per-channel decay:
@@ -410,16 +427,15 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // the decay accumulated since the start of the block, >= 0: it is clamped to kMaxUpExp, and a block where the
     // clamp was hit (a decay of more than 2^100 within 16 tokens in some channel) is evaluated again afterwards,
     // element by element in fp32.
-    int* sFall = reinterpret_cast<int*>(sm + OFF_FALL);
-    if (tid < 4) sFall[tid] = 0;
-    gsync();
     {
-      const int i = tid >> 2, bi16 = i >> 4;
+      // eight threads per token; thread t takes the 8-channel pieces t and t + 8, so that the eight threads of a
+      // token read 256 contiguous bytes of a gate row and a whole 128-byte row of a K / Q tile (no bank conflicts)
+      const int i = tid >> 3, bi16 = i >> 4;
       const int row_k = 32 * bi16 + (i & 15);
       bool clamped = false;
 #pragma unroll 1
-      for (int q = 0; q < 4; ++q) {
-        const int cc = (tid & 3) * 4 + q;
+      for (int q = 0; q < 2; ++q) {
+        const int cc = (tid & 7) + 8 * q;
         const uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
         const uint32_t off = sw128_offset(i, cc & 7);
         float kf[8], qf[8], gi[8], gr[8], t8[8];
@@ -462,16 +478,17 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
-    gsync();
+    bsync();
     // ---- operands rescaled in place: K <- K 2^G (for W), Q <- Q 2^G (for Q~); K e^{G_L - G} for the chain.
     // The tensor cores read the K+ / Q+ / K- copies, not these tiles, so this runs while they work -- unless a
     // diagonal block has to be evaluated again from the raw tiles first.
-    auto rescale_pass = [&]() {
+    auto rescale_pass = [&](bool all_warps) {            // by all 16 warps, or by the first 8 only
     {
-      const int i = tid >> 2;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int cc = (tid & 3) * 4 + q;
+      const int i = all_warps ? tid >> 3 : tid >> 2;
+      const int nq = all_warps ? 2 : 4;
+#pragma unroll 1
+      for (int q = 0; q < nq; ++q) {
+        const int cc = all_warps ? (tid & 7) + 8 * q : (tid & 3) + 4 * q;
         uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
         const uint32_t off = sw128_offset(i, cc & 7);
         float kf[8], qf[8], gi[8], gl[8], kd[8];
@@ -513,7 +530,8 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       umma_commit(bar_mma);
       publish_prev();
     }
-    if (!anyfall) rescale_pass();
+    if (!anyfall) rescale_pass(true);
+    if (is_main) {                                       // the helper warps are done with this item's arithmetic
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
     mph ^= 1;
     gsync();
@@ -554,7 +572,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       // diagonal blocks where the clamp was hit: element by element, 136 pairs (j <= i) per block
       for (int blk = 0; blk < 4; ++blk) {
         if (!sFall[blk]) continue;
-        for (int qq = tid; qq < 136; qq += kPrepThreads) {
+        for (int qq = tid; qq < 136; qq += kPrepThreads) {   // (first 8 warps)
           int il = 0;
           while ((il + 1) * (il + 2) / 2 <= qq) ++il;
           const int jl = qq - il * (il + 1) / 2;
@@ -583,8 +601,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       gsync();                                   // everyone is done with the raw K and Q tiles
-      rescale_pass();
+      rescale_pass(false);
     }
+    }  // is_main
 
   } else {
     // ---- op #1 Gate: inclusive scan of the log-gate over the chunk (warp 1, tokens lane and lane + 32)
@@ -660,6 +679,8 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
   }
+  const long long nxt = cjl + vstride;
+  if (is_main) {                                         // ---- everything down to the Q~ image: the first 8 warps
   gsync();
   PP(5);
 
@@ -824,6 +845,32 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       sc[t] = t < 64 ? __expf(gl - sG[t]) : __expf(gl);
     }
   }
+  }  // is_main
+  // KDA: the helper warps have been waiting here since the gate-dependent passes; the gate matrix was read for
+  // the last time just above and the next item's whereabouts are known: stage its gate rows and betas.
+  if constexpr (KDA) {
+    if (tid == kPrepThreads) {                           // a helper thread works out where the next item is
+      int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
+      bool hn = cjl + vstride < p.total;
+      if (hn) { item_geom(cjl + vstride, jn, jqn, Ln, tok0n); hn = Ln > 0; }
+      sNext[0] = hn ? 1 : 0; sNext[1] = jn; sNext[2] = jqn; sNext[3] = Ln; sNext[4] = tok0n;
+    }
+    bsync();
+    if (sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4]);
+    if (warp == 9) {                                     // another helper warp: the gate rows of the item after
+      int j2 = 0, jq2 = 0, L2 = 0, t2 = 0;               // the next one, into L2 (32 KiB from HBM take a while)
+      if (lane == 0 && cjl + 2 * vstride < p.total) item_geom(cjl + 2 * vstride, j2, jq2, L2, t2);
+      j2 = __shfl_sync(0xffffffffu, j2, 0);
+      L2 = __shfl_sync(0xffffffffu, L2, 0);
+      t2 = __shfl_sync(0xffffffffu, t2, 0);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int t = lane + 32 * h;
+        if (t < L2) bulk_prefetch_l2(p.g + ((size_t)(t2 + t) * p.HV + j2) * 128, 512);
+      }
+    }
+  }
+  if (is_main) {
   if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
   if (tid == 0) bulk_wait_read_1();                      // the W image was read; it receives the Q~ image
   mph ^= 1;
@@ -832,15 +879,18 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   tc_fence_after_sync();
   // Every MMA of this item is done, so the K / Q tile regions are free: start the next item's loads now
   // (its V tiles follow at the top of the loop, once the O_loc image has left their room).
-  const long long nxt = cjl + vstride;
-  if (tid == 0) {                                        // one thread works out where the next item is
-    int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
-    bool hn = nxt < p.total;
-    if (hn) { item_geom(nxt, jn, jqn, Ln, tok0n); hn = Ln > 0; }
-    PP(14);
-    if (hn) issue_tiles(jqn, tok0n);
-    PP(15);
-    sNext[0] = hn ? 1 : 0; sNext[1] = jn; sNext[2] = jqn; sNext[3] = Ln; sNext[4] = tok0n;
+  if (tid == 0) {
+    if constexpr (KDA) {                                 // (a helper thread has worked out where the next item is)
+      if (sNext[0]) issue_tiles(sNext[2], sNext[4]);
+    } else {                                             // one thread works out where the next item is
+      int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
+      bool hn = nxt < p.total;
+      if (hn) { item_geom(nxt, jn, jqn, Ln, tok0n); hn = Ln > 0; }
+      PP(14);
+      if (hn) issue_tiles(jqn, tok0n);
+      PP(15);
+      sNext[0] = hn ? 1 : 0; sNext[1] = jn; sNext[2] = jqn; sNext[3] = Ln; sNext[4] = tok0n;
+    }
   }
   {
     // Q~^T and O_loc^T are complete in the accumulators; their images go where W^T and U^T were.
@@ -855,18 +905,22 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_WT, kImgBytes);
       bulk_commit();
     }
-    if (sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4]);
+    if (!KDA && sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4]);
+  }
+  {
+    float v[32];
     ld32(my_tmem + 64, v);
     store_half_row(v, rowq, hf, sm + OFF_UT);
+    // The accumulators were read: the next item's first MMA may overwrite them after this barrier.
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    gsync();
+    if (tid == 0) {
+      bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
+      bulk_commit();
+    }
   }
-  // The accumulators were read: the next item's first MMA may overwrite them after this barrier.
-  fence_proxy_async_smem();
-  tc_fence_before_sync();
-  gsync();
-  if (tid == 0) {
-    bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
-    bulk_commit();
-  }
+  }  // is_main
   const bool have_n = sNext[0] != 0;
   const int jn = sNext[1], jqn = sNext[2], Ln = sNext[3], tok0n = sNext[4];
   PP(13);
@@ -914,7 +968,7 @@ static cudaError_t launch_prep_variant(const PrepParams& pp, const CUtensorMap& 
                                        const CUtensorMap& mv, long long grid, cudaStream_t stream) {
   const int smem = KDA ? kPrepSmemKda : kGroups<KDA> * kGroupSmem;
   timer_mark(stream, "tc_prep");
-  tc_prep_kernel<KDA><<<(unsigned)grid, kPrepThreads * kGroups<KDA>, smem, stream>>>(mq, mk, mv, pp);
+  tc_prep_kernel<KDA><<<(unsigned)grid, KDA ? kKdaThreads : kPrepThreads * kGroups<KDA>, smem, stream>>>(mq, mk, mv, pp);
   return cudaGetLastError();
 }
 
