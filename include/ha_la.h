@@ -124,7 +124,7 @@ int ha_la_prefill_timed(const ha_la_prefill_args* args, void* cuda_stream, int m
  * counterpart of this entry point; it computes exactly what ha_la_prefill computes.
  *
  *   - args->workspace and args->workspace_bytes are ignored.  The chunk table lives in a fixed
- *     array inside the library image (ha_la_prefill_noalloc_scratch_bytes() bytes, about 208 KiB),
+ *     array inside the library image (ha_la_prefill_noalloc_scratch_bytes() bytes, about 212 KiB),
  *     which every GPU that loads the library holds until the process exits.
  *   - Limits: at most 1024 sequences (batch rows or packed sequences) and at most 16384 chunk
  *     slots ((seqlen + 63 * num_seqs) / 64 in packed mode, batch * ceil(seqlen / 64) otherwise);

@@ -19,6 +19,7 @@ struct PlanView {
   int32_t* seq_tok0;    // [N]   first token row of sequence n
   int32_t* seq_len;     // [N]   tokens in sequence n (0 if the sequence failed a check)
   int32_t* seq_chunk0;  // [N+1] first chunk slot of sequence n (prefix sum)
+  int32_t* seq_order;   // [N]   sequences by descending length (longest first), for launch order
   int32_t* chunk_seq;   // [MC]  sequence of chunk slot s
   int32_t* chunk_tok0;  // [MC]  first token row of chunk slot s
   int32_t* chunk_len;   // [MC]  tokens in chunk slot s (1..64), 0 for an unused slot
@@ -39,7 +40,7 @@ struct Problem {
 inline __host__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 inline __host__ size_t plan_bytes(const Problem& p) {
-  size_t ints = 8 + 2 * (size_t)p.N + ((size_t)p.N + 1) + 3 * (size_t)p.max_chunks;
+  size_t ints = 8 + 3 * (size_t)p.N + ((size_t)p.N + 1) + 3 * (size_t)p.max_chunks;
   return align_up(ints * sizeof(int32_t), 1024);
 }
 
@@ -50,6 +51,7 @@ inline __host__ PlanView plan_view(void* ws, const Problem& p) {
   v.seq_tok0 = b;                  b += p.N;
   v.seq_len = b;                   b += p.N;
   v.seq_chunk0 = b;                b += p.N + 1;
+  v.seq_order = b;                 b += p.N;
   v.chunk_seq = b;                 b += p.max_chunks;
   v.chunk_tok0 = b;                b += p.max_chunks;
   v.chunk_len = b;

@@ -17,8 +17,8 @@ namespace {
 
 constexpr int kMaxSeqs = 1024;        // sequences (batch rows or packed sequences)
 constexpr int kMaxChunks = 16384;     // chunk slots: about one million tokens
-constexpr size_t kScratchInts = 8 + 2 * (size_t)kMaxSeqs + (kMaxSeqs + 1) + 3 * (size_t)kMaxChunks;
-constexpr size_t kScratchBytes = (kScratchInts * sizeof(int32_t) + 255) / 256 * 256;   // 208 KiB
+constexpr size_t kScratchInts = 8 + 3 * (size_t)kMaxSeqs + (kMaxSeqs + 1) + 3 * (size_t)kMaxChunks;
+constexpr size_t kScratchBytes = (kScratchInts * sizeof(int32_t) + 255) / 256 * 256;   // 212 KiB
 
 static __device__ __align__(256) unsigned char g_plan_scratch[kScratchBytes];
 

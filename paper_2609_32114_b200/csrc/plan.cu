@@ -40,6 +40,22 @@ __global__ void __launch_bounds__(256) plan_kernel(PlanParams p, const int32_t* 
   if (tid == 0) s_carry = 0;
   __syncthreads();
 
+  // 1b. sequences by descending length (ties: by index), so that a kernel with one CTA per sequence can start
+  // the longest ones first.  Rank by counting; beyond a few thousand sequences the order is left as it is
+  // (they are then short, and the count would be quadratic).
+  for (int n = tid; n < p.N; n += blockDim.x) {
+    int rank = n;
+    if (p.N <= 4096) {
+      const int len = v.seq_len[n];
+      rank = 0;
+      for (int k = 0; k < p.N; ++k) {
+        const int lk = v.seq_len[k];
+        rank += (lk > len || (lk == len && k < n)) ? 1 : 0;
+      }
+    }
+    v.seq_order[rank] = n;
+  }
+
   // 2. exclusive prefix sum of chunk counts over sequences, 256 at a time
   for (int base = 0; base < p.N; base += blockDim.x) {
     const int n = base + tid;

@@ -69,6 +69,7 @@ int sm_count() {
   return n;
 }
 
+constexpr int kMaxDevices = 64;
 std::atomic<uint32_t> g_calls{0};
 
 // Epoch of a concurrent-mode call: (random per-process tag, never 0) << 32 | call counter.
@@ -83,16 +84,38 @@ int64_t next_epoch() {
 
 // Slice width (value channels per chain CTA) and launch mode.  The chain kernel is bound by the latency of its
 // two MMA round trips per chunk, which grows with the slice width (about 0.9 / 1.4 / 1.95 us per chunk at 32 /
-// 64 / 128 channels on B200) and does not depend on the number of CTAs: take the narrowest slice that still
-// gives every CTA an SM of its own.  Concurrent mode when those CTAs leave at least half of the SMs to the prep
-// kernel and the slice is the narrow one (with 64-channel slices the overlap measured no gain over running
-// the two kernels back to back with 32-channel slices).
+// 64 / 128 channels on B200) and does not depend on the number of CTAs.  Each CTA needs an SM of its own, so
+// the kernel's time is about  max(longest sequence, all sequences / SMs)  in chunk-times when the lengths differ
+// (more CTAs than SMs are started longest sequence first and pack well), and whole rounds when they do not:
+// with few chains the narrow slice wins, with many a wider one may.
+// Only bounds are known on the host: max_len for the longest sequence, max_chunks for the total.
+// Concurrent mode when the CTAs leave at least half of the SMs to the prep kernel and the slice is the narrow
+// one (with 64-channel slices the overlap measured no gain over back-to-back kernels with 32-channel slices).
 struct TcPlan { int nv; bool concurrent; };
 
 TcPlan plan_tc(const Problem& p) {
   const int sms = sm_count();
   const long long chains = (long long)p.N * p.HV;
-  int nv = chains * 4 <= sms ? 32 : (chains * 2 <= sms ? 64 : 128);
+  const double longest = (double)((p.max_len + kChunk - 1) / kChunk);
+  const double items = (double)p.max_chunks * p.HV;
+  const int widths[3] = {32, 64, 128};
+  const double per_chunk_us[3] = {0.90, 1.40, 1.95};
+  int nv = 32;
+  double best = 1e30;
+  // sequences of about the same length (batch rows, or a packed batch whose longest is close to its average)
+  // cannot be packed any better than in rounds of one CTA per SM
+  const double avg_len = p.N > 0 ? (double)p.T_total / p.N : 0.0;
+  const bool even = avg_len <= 0.0 || p.max_len < 1.5 * avg_len;
+  for (int w = 0; w < 3; ++w) {
+    const long long ctas = chains * (128 / widths[w]);
+    const double serial = longest * per_chunk_us[w];
+    double est = serial;
+    if (ctas > sms) {
+      const double spread = 1.15 * items * (128 / widths[w]) * per_chunk_us[w] / sms;
+      est = even ? serial * (double)((ctas + sms - 1) / sms) : (serial > spread ? serial : spread);
+    }
+    if (est < best) { best = est; nv = widths[w]; }
+  }
   if (const char* e = getenv("HA_LA_TC_NV")) {
     const int v = atoi(e);
     if (v == 32 || v == 64 || v == 128) nv = v;
@@ -125,10 +148,18 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   const bool concurrent = tp.concurrent;
   // Configure (and load) both kernels before anything is enqueued: loading a kernel for the first time can
   // wait for the device, and in the concurrent mode the chain kernel would be spinning meanwhile.
-  cudaError_t ce = configure_tc_prep(p);
-  if (ce != cudaSuccess) return ce;
-  ce = configure_tc_chain(p, nv);
-  if (ce != cudaSuccess) return ce;
+  // (Once per device and kernel instance: the attributes stick, and the calls are not free on the host.)
+  static std::atomic<uint32_t> configured[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  const uint32_t bit = 1u << ((p.variant == HA_LA_KDA ? 3 : 0) + (nv == 32 ? 0 : (nv == 64 ? 1 : 2)));
+  if (dev < 0 || dev >= kMaxDevices || !(configured[dev].load() & bit)) {
+    cudaError_t ce = configure_tc_prep(p);
+    if (ce != cudaSuccess) return ce;
+    ce = configure_tc_chain(p, nv);
+    if (ce != cudaSuccess) return ce;
+    if (dev >= 0 && dev < kMaxDevices) configured[dev].fetch_or(bit);
+  }
   int64_t epoch = 0;                                     // 0 means "sequential"
   int reserved_sms = 0;
   if (concurrent) {

@@ -62,6 +62,7 @@ struct ChainParams {
   const int32_t* seq_tok0;     // per-sequence table of the plan kernel, or NULL for equal-length rows
   const int32_t* seq_len;      //   (then sequence n is tokens [n*T_row, (n+1)*T_row), cps chunk slots each)
   const int32_t* seq_chunk0;
+  const int32_t* seq_order;    // launch order of the sequences (longest first), or NULL
   int T_row, cps;
   TcWorkspace ws;
   int HK, HV;
@@ -147,7 +148,8 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   const int warp = tid >> 5;
   const int slice = blockIdx.x % NSL;
   const int nj = blockIdx.x / NSL;
-  const int j = nj % p.HV, n = nj / p.HV;
+  const int j = nj % p.HV;
+  const int n = p.seq_order ? p.seq_order[nj / p.HV] : nj / p.HV;   // CTAs of the longest sequences come first
   const int jq = j / (p.HV / p.HK);
   const int tok0 = p.seq_tok0 ? p.seq_tok0[n] : n * p.T_row;
   const int len = p.seq_tok0 ? p.seq_len[n] : p.T_row;
@@ -417,6 +419,7 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   ChainParams cp;
   cp.h0 = a.h0; cp.hT = a.hT; cp.o = a.o;
   cp.seq_tok0 = plan.seq_tok0; cp.seq_len = plan.seq_len; cp.seq_chunk0 = plan.seq_chunk0;
+  cp.seq_order = plan.seq_tok0 ? plan.seq_order : nullptr;
   cp.T_row = p.T_row; cp.cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
   cp.ws = ws; cp.HK = p.HK; cp.HV = p.HV; cp.scale = p.scale; cp.status = a.status_word;
   cp.epoch = epoch;
