@@ -2,7 +2,7 @@
 // with operator #6 (output) fused in the paper's chunk-first order.
 //
 // One CTA per (sequence, V-head, slice of NV value channels) walks the chunks of its sequence in
-// order.  The d_k x NV slice of the state stays on chip for the whole sequence: fp32 in registers
+// order (there may be more CTAs than SMs; those of the longest sequences come first).  The d_k x NV slice of the state stays on chip for the whole sequence: fp32 in registers
 // (thread t owns key channel t), plus a bf16 copy in shared memory as the MMA operand.  Value
 // channels are independent (paper Section "Computation Splitting": the state splits column-wise
 // into sub-heads with no cross-core reduction), so slices never communicate.
@@ -17,10 +17,11 @@
 // Warp roles: 4 CG compute warps (warp w <-> tensor-memory lanes 32 (w % 4).., column group w / 4 of the
 // slice: CG groups of NV / CG value channels, so that wide slices do not lengthen the epilogues), then one
 // producer warp (keeps the next chunks' operands in flight through a ring of shared-memory stages: 1-D
-// bulk copies + one TMA tile) and one warp that issues the MMAs.  A tcgen05.mma costs the issuing thread about 65 cycles whatever
-// its N <= 128, so issue runs on its own warp and is told "operand ready" with arrive-only named
-// barriers; the compute warps never wait for issue, only for completion (mbarriers).  Every
-// mbarrier wait is bounded.
+// bulk copies + one TMA tile) and one warp that issues the MMAs.  A tcgen05.mma costs the issuing thread
+// some 45-80 cycles whatever its N <= 128, so issue runs on its own warp and is told "operand ready" with
+// arrive-only named barriers; the compute warps never wait for issue, only for completion (mbarriers).
+// In the concurrent mode the producer warp also watches the prep kernel's per-chunk flags (32 at a time).
+// Every mbarrier wait and every flag wait is bounded.
 #include <cuda.h>
 
 #include "tc_common.cuh"

@@ -1,10 +1,14 @@
-// Chunk-local operators of the delta-rule prefill on tcgen05 tensor cores (GDN).
+// Chunk-local operators of the delta-rule prefill on tcgen05 tensor cores (GDN and KDA).
 //
-// One CTA (8 warps) per (chunk slot, V-head).  Implements, for its chunk (paper Section 2.1,
-// "Chunkwise Map-Reduce-Map Execution"):
-//   #1 Gate   G = chunk-local cumulative log-gate (warp scan)
-//   #2 KKT    S = [K; Q] K^T on the tensor cores (one M=128 MMA covers K K^T and Q K^T), then
-//             A_ij = beta_i e^{G_i-G_j} S_kk[i,j] (j<i)  and  P_ij = e^{G_i-G_j} S_qk[i,j] (j<=i) in fp32
+// A persistent kernel, one CTA per SM, whose work items are (chunk slot, V-head) pairs in chunk-major order.
+// GDN: a CTA holds three independent work groups of 8 warps (own shared memory, named barrier and quarter of
+// tensor memory), i.e. three items are in flight per SM.  KDA: one group of 16 warps per CTA; warps 8..15 only
+// run the gate-dependent element-wise passes, stage the next item's gate rows and prefetch later ones into L2.
+// A group implements, for its chunk (paper Section 2.1, "Chunkwise Map-Reduce-Map Execution"):
+//   #1 Gate   G = chunk-local cumulative log-gate (GDN: one scalar per token; KDA: one per key channel)
+//   #2 KKT    GDN: S = [K; Q] K^T on the tensor cores (one M=128 MMA covers K K^T and Q K^T), then
+//             A_ij = beta_i e^{G_i-G_j} S_kk[i,j] (j<i)  and  P_ij = e^{G_i-G_j} S_qk[i,j] (j<=i) in fp32.
+//             KDA: the decay sits inside the contraction; see the comment at that pass.
 //   #3 Solve  T = (I + A)^-1 by blocked forward substitution: four 16x16 diagonal blocks in fp32 registers,
 //             then the off-diagonal blocks level by level as T_lo = -T_hi (A_lo T_lo') on mma.sync (fp16
 //             operands, fp32 accumulation).  A and T are held in shared memory as fp16 (T is rounded to bf16
@@ -15,9 +19,11 @@
 //             Q~ = Q e^G - P W      O_loc = P U        (o = scale [Q~ h + O_loc])
 // (Q e^G enters the Q~ accumulator as one more MMA, Q^T diag(e^G), and P W with the negate-A flag.)
 // Operands arrive by TMA (bf16, 128-byte swizzle), accumulators live in tensor memory, results are
-// assembled in shared memory as ready-to-use operand images (tc_common.cuh) and leave by bulk copy.
+// assembled in shared memory as ready-to-use operand images (tc_common.cuh) and leave by bulk copy.  The next
+// item's tiles, gates and position are fetched while the current one finishes.  When the chain kernel runs
+// concurrently, each item is published with a release flag once its bulk stores have completed.
 //
-// Warp w reads tensor-memory lanes 32*(w%4)..+31 (accumulator rows) and columns 32*(w/4)..+31.
+// Warp w (of the first 8) reads tensor-memory lanes 32*(w%4)..+31 (accumulator rows) and columns 32*(w/4)..+31.
 //
 // Tokens past the end of a sequence are made no-ops by beta = 0 and g = 0; whatever the TMA box
 // read for them (the next sequence's rows, or zero fill past the end of the tensor) is multiplied
