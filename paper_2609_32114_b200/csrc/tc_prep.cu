@@ -878,7 +878,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
   if (is_main) {
   if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
-  if (tid == 0) bulk_wait_read_1();                      // the W image was read; it receives the Q~ image
+  if (tid == 0) bulk_wait_read_all();                    // the W and U images were read; they receive the next two
   mph ^= 1;
   gsync();
   PP(12);
@@ -903,29 +903,19 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     float v[32];
     ld32(my_tmem, v);
     store_half_row(v, rowq, hf, sm + OFF_WT);
-    if (tid == 0) bulk_wait_read_all();                  // the U image was read too
-    fence_proxy_async_smem();
-    tc_fence_before_sync();
-    gsync();
-    if (tid == 0) {
-      bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_WT, kImgBytes);
-      bulk_commit();
-    }
-    if (!KDA && sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4]);
-  }
-  {
-    float v[32];
     ld32(my_tmem + 64, v);
     store_half_row(v, rowq, hf, sm + OFF_UT);
-    // The accumulators were read: the next item's first MMA may overwrite them after this barrier.
-    fence_proxy_async_smem();
-    tc_fence_before_sync();
-    gsync();
-    if (tid == 0) {
-      bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
-      bulk_commit();
-    }
   }
+  // The accumulators were read: the next item's first MMA may overwrite them after this barrier.
+  fence_proxy_async_smem();
+  tc_fence_before_sync();
+  gsync();
+  if (tid == 0) {
+    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_WT, kImgBytes);
+    bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
+    bulk_commit();
+  }
+  if (!KDA && sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4]);   // (after the barrier: thread 0 wrote sNext)
   }  // is_main
   const bool have_n = sNext[0] != 0;
   const int jn = sNext[1], jqn = sNext[2], Ln = sNext[3], tok0n = sNext[4];
