@@ -240,10 +240,12 @@ def main():
     R = max(2, int(np.ceil(2.2 * L2_BYTES / alg_bytes)) + 1)
     R = min(R, 8)
     sets = []
+    shared_ws = None                                     # the workspace is the caller's scratch: one for all sets
     for r in range(R):
         d = base if r == 0 else {k: (v.clone() if hasattr(v, "clone") else v) for k, v in base.items()}
         a, keep = ha.prepare_args(d["q"], d["k"], d["v"], d["g"], d["beta"], variant=w.variant, h0=d["h0"],
-                                  cu_seqlens=d["cu_seqlens"], max_seqlen=d["max_seqlen"])
+                                  cu_seqlens=d["cu_seqlens"], max_seqlen=d["max_seqlen"], workspace=shared_ws)
+        shared_ws = keep["workspace"]
         sets.append((a, keep))
     flush = None
     if R * alg_bytes < 2 * L2_BYTES:
@@ -369,7 +371,7 @@ def main():
                 "config": {"workload": w.name, "variant": w.variant, "tokens_per_step_per_gpu": T, "sequences": N,
                            "seq_lens": inp["seq_lens"] if N <= 16 else None, "qk_heads": w.hk, "v_heads": w.hv,
                            "d_k": w.dk, "d_v": w.dv, "chunk": 64, "path": path,
-                           "l2": f"{R} resident buffer sets visited round-robin ({R * alg_bytes / 1e6:.0f} MB)"
+                           "l2": f"{R} resident input/output sets visited round-robin ({R * alg_bytes / 1e6:.0f} MB), one scratch workspace"
                                  + (" + L2 flush write between steps" if flush is not None else ""),
                            "parallelism": "replicas (independent batch per GPU, no collective)" if world > 1 else "1 GPU"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
