@@ -260,3 +260,44 @@ def test_back_to_back_calls_share_a_workspace():
         assert torch.equal(o, ref[0]) and torch.equal(hT, ref[1]), f"call {it} differs"
     helpers.check_parity(ia)
     helpers.check_parity(ib)
+
+
+def test_two_streams_in_flight():
+    """Calls on two streams at once, each with its own workspace: the prep and chain kernels of the two
+    calls compete for the SMs (together they want more than there are), nothing may deadlock or mix up."""
+    import torch
+    import paper_2609_32114_b200 as ha
+
+    w1 = synth.shrink(W["gdn_layer_4k"], seq_lens=[2048], hk=8, hv=8)
+    w2 = synth.shrink(W["kda_8k"], seq_lens=[1024], hk=4, hv=8)
+    i1, i2 = synth.make_inputs(w1, seed=51), synth.make_inputs(w2, seed=52)
+    d1, d2 = helpers.to_device(i1), helpers.to_device(i2)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+
+    def call(d, w, stream, ws=None):
+        return ha.ha_la_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"], variant=w.variant, h0=d["h0"],
+                                cu_seqlens=d["cu_seqlens"], max_seqlen=d["max_seqlen"], workspace=ws,
+                                stream=stream.cuda_stream)
+
+    ref1 = call(d1, w1, s1)
+    ref2 = call(d2, w2, s2)
+    torch.cuda.synchronize()
+    r1 = (ref1[0].clone(), ref1[1].clone()); r2 = (ref2[0].clone(), ref2[1].clone())
+    ws1, ws2 = ref1[3], ref2[3]
+    outs = []
+    for it in range(6):
+        a = call(d1, w1, s1, ws1)
+        b = call(d2, w2, s2, ws2)
+        with torch.cuda.stream(s1):
+            oa = (a[0].clone(), a[1].clone(), a[2])
+        with torch.cuda.stream(s2):
+            ob = (b[0].clone(), b[1].clone(), b[2])
+        outs.append((oa, ob))
+    torch.cuda.synchronize()
+    for oa, ob in outs:
+        assert int(oa[2].item()) == 0 and int(ob[2].item()) == 0
+        assert torch.equal(oa[0], r1[0]) and torch.equal(oa[1], r1[1])
+        assert torch.equal(ob[0], r2[0]) and torch.equal(ob[1], r2[1])
+    helpers.check_parity(i1)
+    helpers.check_parity(i2)
