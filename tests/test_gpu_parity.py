@@ -301,3 +301,18 @@ def test_two_streams_in_flight():
         assert torch.equal(ob[0], r2[0]) and torch.equal(ob[1], r2[1])
     helpers.check_parity(i1)
     helpers.check_parity(i2)
+
+
+@pytest.mark.parametrize("variant", ["gdn", "kda"])
+def test_many_sequences_more_ctas_than_sms(variant):
+    """A packed batch with many (sequence, V-head) chains of very different lengths: the chain kernel then
+    has more CTAs than the GPU has SMs and starts them longest sequence first."""
+    rng = np.random.default_rng(5)
+    lens = [int(x) for x in rng.integers(1, 900, size=90)]
+    lens[7] = 0
+    lens[40] = 2500
+    base = W["gdn_varlen"] if variant == "gdn" else W["kda_8k"]
+    w = synth.shrink(base, seq_lens=lens, hk=2, hv=4, h0_std=0.02, varlen=True)
+    inp = synth.make_inputs(w, seed=61)
+    res = helpers.check_parity(inp, scale=0.5)
+    print(variant, res)
