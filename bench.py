@@ -76,7 +76,6 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=2)
@@ -299,7 +298,17 @@ def main():
             flush.fill_(i)
         for name, ms in ha.ha_la_prefill_timed(sets[(i + 1) % R][0], sptr):
             kt.setdefault(name, []).append(ms)
+    # nvidia-smi cannot sample faster than every ~100 ms and a timed region of K short steps is over before
+    # its first sample: keep the same steps running (untimed) until a few samples have been taken under this load.
+    t_load = time.perf_counter()
+    i = 0
+    while len(sampler.rows) < 4 and time.perf_counter() - t_load < 2.0:
+        for _ in range(16):
+            step(i)
+            i += 1
+        barrier()
     clocks = sampler.stop()
+    clocks["window"] = f"timed region, per-kernel timing and {time.perf_counter() - t_load:.2f} s of the same steps"
     kernel_ms = {k: float(np.mean(v)) for k, v in kt.items()}
     dom = max(kernel_ms, key=kernel_ms.get)
     # algorithmic bytes each kernel is the one to touch ("Roofline accounting")
