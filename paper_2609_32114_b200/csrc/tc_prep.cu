@@ -377,6 +377,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (tid == 0) {
       if (prev_cj >= 0) bulk_wait_read_all();
       issue_v(j, tok0);
+      publish_prev();
     }
     bsync();
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
@@ -534,7 +535,6 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       umma_commit(bar_mma);
-      publish_prev();
     }
     if (!anyfall) rescale_pass(true);
     if (is_main) {                                       // the helper warps are done with this item's arithmetic
@@ -635,6 +635,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ---- op #2 KKT (+ Q K^T): S[0:64] = K K^T, S[64:128] = Q K^T
     if (tid == 0) {
       PP(2);
+      publish_prev();                                    // (its wait for the stores overlaps the tiles' arrival)
       mbar_wait(bar_load, lph, abort_flag);
       PP(3);
       // the previous item's W / U images must have left before V lands on one and A is written over the other
@@ -649,7 +650,6 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         umma_ss(tmem, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(a, 16, 1024, kSwizzle128B), id, ks > 0);
       }
       umma_commit(bar_mma);
-      publish_prev();
     }
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);  // one warp polls; the others sleep at the barrier
     mph ^= 1;
