@@ -37,6 +37,9 @@
  *     with unspecified outputs.
  *   - o must not overlap any input.  hT may be exactly the pointer h0
  *     (in-place state update) and must not partially overlap it.
+ *   - The workspace is scratch for ONE call at a time: its contents on entry do
+ *     not matter and nothing in it needs clearing, but calls that may overlap on
+ *     the GPU (different streams without an ordering) need a workspace each.
  *   - Sequence lengths need not be multiples of 64; length-0 sequences are
  *     legal (hT = h0).  Log-gates are expected to be <= 0.
  */
