@@ -144,6 +144,41 @@ int ha_la_prefill_timed(const ha_la_prefill_args* args, void* cuda_stream, int m
 int ha_la_prefill_noalloc(const ha_la_prefill_args* args, void* cuda_stream);
 size_t ha_la_prefill_noalloc_scratch_bytes(void);
 
+/* One decoding step of the same layer: ONE new token per sequence, the recurrent state kept by the
+ * caller between calls.  The paper hands "updated states for downstream layers and subsequent
+ * decoding" from the prefill to the decoder (Section "HA-NPU overview") and leaves the decoding
+ * step itself to the framework's native backend; this entry point is that step for the state
+ * layout ha_la_prefill produces (hT), so that prefill and decode share one library.
+ *
+ * For every sequence n and V-head j (QK-head jq = j / (HV/HK)), with h = h_in[n,j] (zeros if NULL):
+ *     GDN:  h <- exp(g[n,j]) h            KDA:  h[c,:] <- exp(g[n,j,c]) h[c,:]
+ *     h <- h + beta[n,j] k[n,jq] (v[n,j] - h^T k[n,jq])^T
+ *     o[n,j] = scale * h^T q[n,jq]         h_out[n,j] = h
+ * All arithmetic is fp32.  Device pointers, asynchronous on the stream, no workspace, no allocation.
+ * q, k, v, o, h_in, h_out 16-byte aligned; h_out may be exactly h_in (in place) and must not
+ * partially overlap it; o must not overlap any input.                                             */
+typedef struct {
+  int32_t variant;        /* ha_la_variant                                                   */
+  int32_t dtype;          /* ha_la_dtype of q, k, v and o                                    */
+  int32_t num_seqs;       /* N >= 0: sequences, one token each                               */
+  int32_t num_qk_heads;   /* HK                                                              */
+  int32_t num_v_heads;    /* HV, a multiple of HK                                            */
+  int32_t d_k, d_v;       /* d_k == d_v, 64 or 128                                           */
+  float   scale;
+  const void*  q;         /* [N, HK, d_k]                                                    */
+  const void*  k;         /* [N, HK, d_k]                                                    */
+  const void*  v;         /* [N, HV, d_v]                                                    */
+  const float* g;         /* GDN [N, HV]; KDA [N, HV, d_k]; log-gate                         */
+  const float* beta;      /* [N, HV]                                                         */
+  const float* h_in;      /* [N, HV, d_k, d_v] fp32 or NULL (zeros)                          */
+  float*       h_out;     /* [N, HV, d_k, d_v] fp32                                          */
+  void*        o;         /* [N, HV, d_v], dtype as v                                        */
+} ha_la_decode_args;
+
+/* Enqueue one decoding step on `cuda_stream`.  Returns HA_LA_OK or an error code; launches one
+ * kernel (none when N == 0).                                                                      */
+int ha_la_decode(const ha_la_decode_args* args, void* cuda_stream);
+
 const char* ha_la_status_string(int status);
 int ha_la_version(void);
 

@@ -7,6 +7,9 @@ library has not been built.
 """
 from .binding import (  # noqa: F401
     HaLaError,
+    ha_la_decode,
+    ha_la_decode_args,
+    ha_la_decode_raw,
     ha_la_prefill,
     ha_la_prefill_args,
     ha_la_prefill_num_launches,
@@ -20,5 +23,6 @@ from .binding import (  # noqa: F401
     load_library,
     make_args,
     prepare_args,
+    prepare_decode_args,
     status_string,
 )

@@ -31,6 +31,7 @@ EXPORTS = (
     "ha_la_prefill_noalloc_scratch_bytes",
     "ha_la_prefill_path",
     "ha_la_prefill_num_launches",
+    "ha_la_decode",
     "ha_la_status_string",
     "ha_la_version",
 )
@@ -62,6 +63,27 @@ class ha_la_prefill_args(ctypes.Structure):
         ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t),
         ("status_word", ctypes.c_void_p),
+    ]
+
+
+class ha_la_decode_args(ctypes.Structure):
+    _fields_ = [
+        ("variant", ctypes.c_int32),
+        ("dtype", ctypes.c_int32),
+        ("num_seqs", ctypes.c_int32),
+        ("num_qk_heads", ctypes.c_int32),
+        ("num_v_heads", ctypes.c_int32),
+        ("d_k", ctypes.c_int32),
+        ("d_v", ctypes.c_int32),
+        ("scale", ctypes.c_float),
+        ("q", ctypes.c_void_p),
+        ("k", ctypes.c_void_p),
+        ("v", ctypes.c_void_p),
+        ("g", ctypes.c_void_p),
+        ("beta", ctypes.c_void_p),
+        ("h_in", ctypes.c_void_p),
+        ("h_out", ctypes.c_void_p),
+        ("o", ctypes.c_void_p),
     ]
 
 
@@ -101,6 +123,8 @@ def load_library(path: Optional[str] = None):
     lib.ha_la_prefill_path.restype = ctypes.c_char_p
     lib.ha_la_prefill_num_launches.argtypes = [A]
     lib.ha_la_prefill_num_launches.restype = ctypes.c_int
+    lib.ha_la_decode.argtypes = [ctypes.POINTER(ha_la_decode_args), ctypes.c_void_p]
+    lib.ha_la_decode.restype = ctypes.c_int
     lib.ha_la_status_string.argtypes = [ctypes.c_int]
     lib.ha_la_status_string.restype = ctypes.c_char_p
     lib.ha_la_version.argtypes = []
@@ -237,3 +261,41 @@ def ha_la_prefill(q, k, v, g, beta, *, stream=None, **kw):
         raise HaLaError(rc, "ha_la_prefill")
     o = keep["o"].squeeze(0) if squeeze else keep["o"]
     return o, keep["hT"], keep["status_word"], keep["workspace"]
+
+
+def prepare_decode_args(q, k, v, g, beta, state, *, variant="gdn", scale=1.0, o=None, state_out=None):
+    """Marshal torch CUDA tensors into ha_la_decode_args.  q, k: [N, HK, d]; v: [N, HV, d]; g: fp32 [N, HV] (gdn)
+    or [N, HV, d] (kda); beta: fp32 [N, HV]; state: fp32 [N, HV, d, d] or None (zeros).  The new state goes to
+    `state_out` (default: in place into `state`; allocated when `state` is None)."""
+    import torch
+
+    N, HK, d = q.shape
+    HV = v.shape[1]
+    if o is None:
+        o = torch.empty_like(v)
+    if state_out is None:
+        state_out = state if state is not None else torch.empty(N, HV, d, d, dtype=torch.float32, device=q.device)
+    ptr = lambda t: t.data_ptr() if t is not None else None
+    args = ha_la_decode_args(variant=0 if variant == "gdn" else 1, dtype=0 if q.dtype == torch.bfloat16 else 1,
+                             num_seqs=N, num_qk_heads=HK, num_v_heads=HV, d_k=d, d_v=v.shape[2], scale=scale,
+                             q=ptr(q), k=ptr(k), v=ptr(v), g=ptr(g), beta=ptr(beta), h_in=ptr(state),
+                             h_out=ptr(state_out), o=ptr(o))
+    return args, dict(q=q, k=k, v=v, g=g, beta=beta, state=state, state_out=state_out, o=o)
+
+
+def ha_la_decode_raw(args: ha_la_decode_args, stream: int = 0) -> int:
+    return load_library().ha_la_decode(ctypes.byref(args), ctypes.c_void_p(stream))
+
+
+def ha_la_decode(q, k, v, g, beta, state, *, stream=None, **kw):
+    """One decoding step on torch CUDA tensors (see prepare_decode_args).  Returns (o, new_state); nothing is
+    synchronised."""
+    import torch
+
+    args, keep = prepare_decode_args(q, k, v, g, beta, state, **kw)
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    rc = ha_la_decode_raw(args, stream)
+    if rc != HA_LA_OK:
+        raise HaLaError(rc, "ha_la_decode")
+    return keep["o"], keep["state_out"]

@@ -21,7 +21,7 @@ INCLUDE = os.path.join(ROOT, "include")
 
 # (object name, source, extra flags)
 UNITS = [("api", "api.cu", []), ("plan", "plan.cu", []), ("tc", "tc.cu", []), ("tc_prep", "tc_prep.cu", []), ("tc_chain", "tc_chain.cu", []),
-         ("noalloc", "noalloc.cu", [])] + [
+         ("noalloc", "noalloc.cu", []), ("decode", "decode.cu", [])] + [
     (f"simt{u}", "simt.cu", [f"-DHA_LA_SIMT_UNIT={u}"]) for u in range(5)
 ]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
