@@ -192,12 +192,177 @@ def job_throughput(world: int, tokens_per_rank: int, ms_per_step: float) -> floa
     return world * tokens_per_rank / (ms_per_step / 1e3)
 
 
+# ---- the decoding step (one new token per sequence on the prefill's state layout): an extra measured row, not
+# the headline metric.  Batch of sequences x heads of the headline layer; the fp32 states (268 MB) exceed L2.
+DECODE_WORKLOADS = {"gdn_decode_b256": ("gdn", 256, 16, 16, 128), "kda_decode_b256": ("kda", 256, 16, 16, 128)}
+
+
+def decode_bench(args, rank, local_rank, world):
+    variant, N, hk, hv, d = DECODE_WORKLOADS[args.workload]
+    base = synth.WORKLOADS["gdn_varlen" if variant == "gdn" else "kda_8k"]
+    w = synth.shrink(base, seq_lens=[1] * N, hk=hk, hv=hv, dk=d, dv=d, dtype="bf16", h0_std=0.5, varlen=True)
+    inp = synth.make_inputs(w, seed=rank_seed(rank))
+    # bytes one step must move: state in and out, q k v g beta in, o out
+    state_bytes = N * hv * d * d * 4
+    io_bytes = N * (2 * hk * d * 2 + 2 * hv * d * 2 + hv * 4 * (1 + (d if variant == "kda" else 1)))
+    alg_bytes = 2 * state_bytes + io_bytes
+    alg_flops = N * hv * 6.0 * d * d
+    metric = "LA-layer decode tokens/s"
+
+    def oracle_run():
+        import oracle
+        t0 = time.perf_counter()
+        _, _, threads = oracle.recurrent(inp["q"], inp["k"], inp["v"], inp["g"], inp["beta"], variant=variant,
+                                         h0=inp["h0"], cu_seqlens=inp["cu_seqlens"])
+        return time.perf_counter() - t0, threads
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        for _ in range(max(args.warmup, 1)):
+            oracle_run()
+        ts = [oracle_run() for _ in range(args.steps)]
+        sec = float(np.mean([t for t, _ in ts]))
+        val = N / sec
+        cpu = {"value": val, "unit": "tokens/s", "cores": ts[0][1], "kind": "oracle",
+               "sample": f"all {N} sequences x {hv} V-heads, one token each"}
+        print(json.dumps({"impl": "reference", "metric": metric, "value": val, "unit": "tokens/s", "n_gpus": world,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                          "data": "synthetic", "config": {"workload": args.workload}, "cpu_baseline": cpu,
+                          "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0,
+                                  "d2h_bytes_per_step": 0}}), flush=True)
+        return
+
+    import torch
+    import paper_2609_32114_b200 as ha
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dev).to(dt).contiguous()
+    bf, f32 = torch.bfloat16, torch.float32
+    q, k, v = t(inp["q"], bf), t(inp["k"], bf), t(inp["v"], bf)
+    g, beta, state = t(inp["g"], f32), t(inp["beta"], f32), t(inp["h0"], f32)
+    dargs, keep = ha.prepare_decode_args(q, k, v, g, beta, state, variant=variant)
+    stream = torch.cuda.current_stream(dev)
+    sptr = stream.cuda_stream
+
+    def step():
+        rc = ha.ha_la_decode_raw(dargs, sptr)
+        if rc != 0:
+            raise ha.HaLaError(rc, "ha_la_decode")
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    t_wall = time.perf_counter()
+    for i in range(args.steps):
+        evs[i][0].record(stream)
+        step()
+        evs[i][1].record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    total_ms = max_over_ranks(dist, float(np.sum([a.elapsed_time(b) for a, b in evs])), dev)
+    ms_per_step = total_ms / args.steps
+    t_load = time.perf_counter()
+    while len(sampler.rows) < 4 and time.perf_counter() - t_load < 2.0:
+        for _ in range(64):
+            step()
+        barrier()
+    clocks = sampler.stop()
+    clocks["window"] = f"timed region and {time.perf_counter() - t_load:.2f} s of the same steps"
+
+    # end to end: the state stays on the device (that is the point of a decoder), the token's inputs come from
+    # pinned host memory and its outputs go back, every step
+    names = ("q", "k", "v", "g", "beta")
+    host = {n_: keep[n_].cpu().pin_memory() for n_ in names}
+    o_host = torch.empty_like(keep["o"], device="cpu").pin_memory()
+    h2d = sum(host[n_].numel() * host[n_].element_size() for n_ in names)
+    d2h = o_host.numel() * o_host.element_size()
+
+    def e2e_step():
+        for n_ in names:
+            keep[n_].copy_(host[n_], non_blocking=True)
+        step()
+        o_host.copy_(keep["o"], non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(dist, e0.elapsed_time(e1), dev)
+    peaks = load_peaks()
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        oracle_run()
+        reps, tot, thr = 0, 0.0, 0
+        while tot * max(thr, 1) < 12.0 and reps < 200:
+            sec, thr = oracle_run()
+            tot += sec
+            reps += 1
+        cpu = {"value": N * reps / tot, "unit": "tokens/s", "cores": thr, "kind": "oracle",
+               "sample": f"all {N} sequences x {hv} V-heads, one token each; {reps} repetition(s), {tot:.2f} s wall"}
+    if rank == 0:
+        sec = ms_per_step / 1e3
+        achieved = alg_bytes / sec / 1e9
+        roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                    "traffic": DECODE_NCU_TRAFFIC.get(args.workload), "kernel_alg_bytes": alg_bytes,
+                    "peak_source": peaks["source"], "kernel_ms": {"decode_kernel": ms_per_step},
+                    "path": {"bound": "hbm", "roofline_us": 1e6 * alg_bytes / (peaks["hbm_gbs"] * 1e9),
+                             "measured_us": 1e3 * ms_per_step, "frac": achieved / peaks["hbm_gbs"],
+                             "achieved_gbs": achieved, "achieved_tflops": alg_flops / sec / 1e12,
+                             "alg_bytes": alg_bytes, "alg_flops": alg_flops}}
+        print(json.dumps({
+            "metric": metric, "value": job_throughput(world, N, ms_per_step), "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "variant": variant, "sequences": N, "qk_heads": hk, "v_heads": hv,
+                       "d_k": d, "d_v": d, "state_bytes": state_bytes,
+                       "l2": "the states (read and rewritten in place every step) exceed L2",
+                       "parallelism": "replicas (independent batch per GPU, no collective)" if world > 1 else "1 GPU"},
+            "clocks": clocks,
+            "e2e": {"value": job_throughput(world, N, e2e_ms / args.steps), "unit": "tokens/s",
+                    "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "mode": "states resident on the device; the token's inputs in and outputs out every step"},
+            "gpu_launches": args.steps, "roofline": roofline, "cpu_baseline": cpu,
+            "wall_s_timed_region": t_wall}), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# DRAM bytes per launch of the decode kernel from its ncu capture (profiles/decode_gdn_decode_b256_ncu_full.md)
+DECODE_NCU_TRAFFIC = {"gdn_decode_b256": 271.64e6 + 212.57e6}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="gdn_layer_4k", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default="gdn_layer_4k", choices=sorted(synth.WORKLOADS) + sorted(DECODE_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -207,6 +372,8 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
+    if args.workload in DECODE_WORKLOADS:
+        return decode_bench(args, rank, local_rank, world)
     w = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
         if rank == 0:

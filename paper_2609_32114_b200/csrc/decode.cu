@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(D) decode_kernel(DecodeParams p) {
   float h[D];
   const float* hin = p.h_in ? p.h_in + nj * D * D + tid : nullptr;
 #pragma unroll
-  for (int c = 0; c < D; ++c) h[c] = hin ? hin[(size_t)c * D] : 0.f;
+  for (int c = 0; c < D; ++c) h[c] = hin ? __ldcs(hin + (size_t)c * D) : 0.f;   // streaming: read once
   __syncthreads();
 
   float r = 0.f;                                         // (decayed h)^T k
@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(D) decode_kernel(DecodeParams p) {
   for (int c = 0; c < D; ++c) {
     h[c] = fmaf(sk[c], u, h[c]);
     acc = fmaf(h[c], sq[c], acc);
-    hout[(size_t)c * D] = h[c];
+    __stcs(hout + (size_t)c * D, h[c]);
   }
   reinterpret_cast<In*>(p.o)[nj * D + tid] = from_f32<In>(p.scale * acc);
 }
