@@ -76,6 +76,28 @@ def test_single_token_closed_form(variant):
     assert abs(kq) > 1e-3 and np.abs(o0).max() > 0     # the output uses the UPDATED state
 
 
+@pytest.mark.parametrize("variant", ["gdn", "kda"])
+def test_decode_step_closed_form_batched(variant):
+    """The decoding step is the recurrence on sequences of length one with the state as h0: a packed batch of
+    N such sequences (grouped values, HV = 2 HK) equals the single-token closed form per (sequence, V-head),
+    and the new state equals decay(h0) + beta k (v - decay(h0)^T k)^T written out."""
+    rng = np.random.default_rng(11)
+    N, hk, hv, dk, dv = 5, 2, 4, 6, 6
+    q, k, v, g, beta = _rand(rng, N, hk, hv, dk, dv, variant, unit_keys=False)
+    h0 = rng.standard_normal((N, hv, dk, dv)).astype(np.float32)
+    cu = np.arange(N + 1, dtype=np.int32)
+    o, hT, _ = oracle.recurrent(q, k, v, g, beta, variant=variant, h0=h0, cu_seqlens=cu, scale=1.3)
+    for n in range(N):
+        for j in range(hv):
+            jq = j // (hv // hk)
+            qq, kk, vv, b = _d(q[n, jq]), _d(k[n, jq]), _d(v[n, j]), float(beta[n, j])
+            dec = np.exp(_d(g[n, j])) * np.ones(dk)
+            hd = dec[:, None] * _d(h0[n, j])
+            hnew = hd + b * np.outer(kk, vv - hd.T @ kk)
+            np.testing.assert_allclose(hT[n, j], hnew, rtol=1e-12, atol=1e-13)
+            np.testing.assert_allclose(o[n, j], 1.3 * (hnew.T @ qq), rtol=1e-12, atol=1e-13)
+
+
 # ---------------------------------------------------------------- matrix form of the recurrence
 
 @pytest.mark.parametrize("variant", ["gdn", "kda"])
