@@ -354,7 +354,7 @@ def decode_bench(args, rank, local_rank, world):
 
 
 # DRAM bytes per launch of the decode kernel from its ncu capture (profiles/decode_gdn_decode_b256_ncu_full.md)
-DECODE_NCU_TRAFFIC = {"gdn_decode_b256": 271.64e6 + 212.57e6}
+DECODE_NCU_TRAFFIC = {"gdn_decode_b256": 271.69e6 + 211.84e6}
 
 
 def main():

@@ -2,9 +2,10 @@
 //
 // The step reads and rewrites the whole fp32 state (d_k x d_v per sequence and V-head, 64 KiB at d = 128) for
 // about 6 d_k d_v flops, so it is bound by HBM traffic: 2 x 4 d_k d_v bytes per (sequence, V-head).  One CTA
-// per (sequence, V-head), one thread per value channel: a thread keeps its column of the state in registers
-// (d_k values), so the state crosses the memory system exactly once in each direction, with every load and
-// store of a warp covering 128 contiguous bytes and all d_k loads of a thread independent (in flight together).
+// per (sequence, V-head), one or two threads per value channel: a thread keeps (half of) its column of the state
+// in registers, so the state crosses the memory system exactly once in each direction, with every load and
+// store of a warp covering 128 contiguous bytes and all loads of a thread independent (in flight together);
+// the state is read and written with streaming hints (it is used once per step and exceeds L2).
 #include "common.cuh"
 
 #include <cuda_bf16.h>
@@ -28,51 +29,78 @@ template <typename T> __device__ __forceinline__ T from_f32(float x);
 template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
-template <typename In, int D, bool KDA>
-__global__ void __launch_bounds__(D) decode_kernel(DecodeParams p) {
-  __shared__ __align__(16) float sk[D];                  // k, then q, then the per-row decay
+// R threads share a column of the state (R = 2 at d = 128: 64 rows and 64 registers each, which lets four
+// CTAs instead of two be resident per SM; the two partial dot products meet in shared memory).
+template <typename In, int D, bool KDA, int R>
+__global__ void __launch_bounds__(D * R) decode_kernel(DecodeParams p) {
+  constexpr int ROWS = D / R;
+  __shared__ __align__(16) float sk[D];
   __shared__ __align__(16) float sq[D];
   __shared__ __align__(16) float sdec[D];
+  __shared__ float spart[R][D];
   const int tid = threadIdx.x;
+  const int col = tid % D, part = tid / D;               // value channel, which block of rows
   const size_t nj = blockIdx.x;                          // (sequence, V-head)
   const int j = (int)(nj % p.HV);
   const size_t n = nj / p.HV;
   const int jq = j / (p.HV / p.HK);
-  const size_t qk_off = (n * p.HK + jq) * D + tid;
-  sk[tid] = to_f32(reinterpret_cast<const In*>(p.k)[qk_off]);
-  sq[tid] = to_f32(reinterpret_cast<const In*>(p.q)[qk_off]);
-  sdec[tid] = __expf(KDA ? p.g[nj * D + tid] : p.g[nj]);
-  const float vv = to_f32(reinterpret_cast<const In*>(p.v)[nj * D + tid]);
+  if (part == 0) {
+    const size_t qk_off = (n * p.HK + jq) * D + col;
+    sk[col] = to_f32(reinterpret_cast<const In*>(p.k)[qk_off]);
+    sq[col] = to_f32(reinterpret_cast<const In*>(p.q)[qk_off]);
+    sdec[col] = __expf(KDA ? p.g[nj * D + col] : p.g[nj]);
+  }
+  const float vv = to_f32(reinterpret_cast<const In*>(p.v)[nj * D + col]);
   const float beta = p.beta[nj];
 
-  // column `tid` of the state, all d_k rows; the loads do not depend on anything above
-  float h[D];
-  const float* hin = p.h_in ? p.h_in + nj * D * D + tid : nullptr;
+  // rows part*ROWS .. of column `col`; the loads do not depend on anything above and are read exactly once
+  float h[ROWS];
+  const size_t base = nj * D * D + (size_t)part * ROWS * D + col;
+  const float* hin = p.h_in ? p.h_in + base : nullptr;
 #pragma unroll
-  for (int c = 0; c < D; ++c) h[c] = hin ? __ldcs(hin + (size_t)c * D) : 0.f;   // streaming: read once
+  for (int c = 0; c < ROWS; ++c) h[c] = hin ? __ldcs(hin + (size_t)c * D) : 0.f;
   __syncthreads();
 
-  float r = 0.f;                                         // (decayed h)^T k
+  const float* k_ = sk + part * ROWS;
+  const float* q_ = sq + part * ROWS;
+  const float* dec_ = sdec + part * ROWS;
+  float r = 0.f;                                         // (decayed h)^T k, this thread's rows
 #pragma unroll
-  for (int c = 0; c < D; ++c) {
-    h[c] *= sdec[c];
-    r = fmaf(h[c], sk[c], r);
+  for (int c = 0; c < ROWS; ++c) {
+    h[c] *= dec_[c];
+    r = fmaf(h[c], k_[c], r);
+  }
+  if (R > 1) {
+    spart[part][col] = r;
+    __syncthreads();
+    r = 0.f;
+#pragma unroll
+    for (int pp = 0; pp < R; ++pp) r += spart[pp][col];
+    __syncthreads();
   }
   const float u = beta * (vv - r);
   float acc = 0.f;
-  float* hout = p.h_out + nj * D * D + tid;
+  float* hout = p.h_out + base;
 #pragma unroll
-  for (int c = 0; c < D; ++c) {
-    h[c] = fmaf(sk[c], u, h[c]);
-    acc = fmaf(h[c], sq[c], acc);
+  for (int c = 0; c < ROWS; ++c) {
+    h[c] = fmaf(k_[c], u, h[c]);
+    acc = fmaf(h[c], q_[c], acc);
     __stcs(hout + (size_t)c * D, h[c]);
   }
-  reinterpret_cast<In*>(p.o)[nj * D + tid] = from_f32<In>(p.scale * acc);
+  if (R > 1) {
+    spart[part][col] = acc;
+    __syncthreads();
+    acc = 0.f;
+#pragma unroll
+    for (int pp = 0; pp < R; ++pp) acc += spart[pp][col];
+  }
+  if (part == 0) reinterpret_cast<In*>(p.o)[nj * D + col] = from_f32<In>(p.scale * acc);
 }
 
 template <typename In, int D, bool KDA>
 cudaError_t launch(const DecodeParams& dp, size_t grid, cudaStream_t stream) {
-  decode_kernel<In, D, KDA><<<(unsigned)grid, D, 0, stream>>>(dp);
+  constexpr int R = D == 128 ? 2 : 1;
+  decode_kernel<In, D, KDA, R><<<(unsigned)grid, D * R, 0, stream>>>(dp);
   return cudaGetLastError();
 }
 
