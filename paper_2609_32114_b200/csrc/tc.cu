@@ -23,7 +23,8 @@ cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanVi
                            const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, int64_t epoch,
                            int reserved_sms, cudaStream_t stream);
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                            const CUtensorMap& mk, int nv, int64_t epoch, bool dependent, cudaStream_t stream);
+                            const CUtensorMap& mk, const CUtensorMap& mo, int nv, int64_t epoch, bool dependent,
+                            cudaStream_t stream);
 
 cudaError_t configure_tc_prep(const Problem& p);
 cudaError_t configure_tc_chain(const Problem& p, int nv);
@@ -59,6 +60,20 @@ bool make_map(CUtensorMap* m, const void* base, int T, int H) {
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The output o as the chain kernel stores it: box = one slice block (nv <= 64 channels) x 1 head x 64 tokens,
+// swizzled like the kernel's staging tile.  Store coordinates are multiples of 32 channels (64 bytes).
+bool make_map_o(CUtensorMap* m, const void* base, int T, int H, int nv) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return false;
+  const cuuint64_t dims[3] = {128, (cuuint64_t)H, (cuuint64_t)(T > 0 ? T : 1)};
+  const cuuint64_t strides[2] = {128 * 2, (cuuint64_t)H * 128 * 2};
+  const cuuint32_t box[3] = {(cuuint32_t)(nv < 64 ? nv : 64), 1, 64};
+  const cuuint32_t es[3] = {1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, nv < 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int sm_count() {
   static int n = [] {
     int dev = 0, v = 0;
@@ -83,7 +98,7 @@ int64_t next_epoch() {
 }
 
 // Slice width (value channels per chain CTA) and launch mode.  The chain kernel is bound by the latency of its
-// two MMA round trips per chunk, which grows with the slice width (about 0.9 / 1.4 / 1.95 us per chunk at 32 /
+// two MMA round trips per chunk, which grows with the slice width (about 0.9 / 1.23 / 1.7 us per chunk at 32 /
 // 64 / 128 channels on B200) and does not depend on the number of CTAs.  Each CTA needs an SM of its own, so
 // the kernel's time is about  max(longest sequence, all sequences / SMs)  in chunk-times when the lengths differ
 // (more CTAs than SMs are started longest sequence first and pack well), and whole rounds when they do not:
@@ -99,7 +114,7 @@ TcPlan plan_tc(const Problem& p) {
   const double longest = (double)((p.max_len + kChunk - 1) / kChunk);
   const double items = (double)p.max_chunks * p.HV;
   const int widths[3] = {32, 64, 128};
-  const double per_chunk_us[3] = {0.90, 1.40, 1.95};
+  const double per_chunk_us[3] = {0.90, 1.23, 1.70};
   int nv = 32;
   double best = 1e30;
   // sequences of about the same length (batch rows, or a packed batch whose longest is close to its average)
@@ -138,13 +153,13 @@ size_t tc_workspace_bytes(const Problem& p) {
 int tc_num_launches(const Problem&) { return 2; }
 
 cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView plan, void* tc_ws, cudaStream_t stream) {
-  CUtensorMap mq, mk, mv;
-  if (!make_map(&mq, a.q, p.T_total, p.HK) || !make_map(&mk, a.k, p.T_total, p.HK) ||
-      !make_map(&mv, a.v, p.T_total, p.HV))
-    return cudaErrorInvalidValue;
-  const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
   const TcPlan tp = plan_tc(p);
   const int nv = tp.nv;
+  CUtensorMap mq, mk, mv, mo;
+  if (!make_map(&mq, a.q, p.T_total, p.HK) || !make_map(&mk, a.k, p.T_total, p.HK) ||
+      !make_map(&mv, a.v, p.T_total, p.HV) || !make_map_o(&mo, a.o, p.T_total, p.HV, nv))
+    return cudaErrorInvalidValue;
+  const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
   const bool concurrent = tp.concurrent;
   // Configure (and load) both kernels before anything is enqueued: loading a kernel for the first time can
   // wait for the device, and in the concurrent mode the chain kernel would be spinning meanwhile.
@@ -168,7 +183,7 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   }
   cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, reserved_sms, stream);
   if (e != cudaSuccess) return e;
-  return launch_tc_chain(p, a, plan, ws, mk, nv, epoch, /*dependent=*/g_timer == nullptr, stream);
+  return launch_tc_chain(p, a, plan, ws, mk, mo, nv, epoch, /*dependent=*/g_timer == nullptr, stream);
 }
 
 }  // namespace ha_la

@@ -51,8 +51,10 @@ template <int NV, int S_> struct ChainCfg {
   static constexpr uint32_t kTxBytes = 32768 + 16384 + 2 * kSliceB + 768;
   static constexpr uint32_t OFF_H = kStages * kStageB;           // bf16 h operand [128][NV]
   static constexpr uint32_t OFF_UT = OFF_H + 128 * kRowB;        // bf16 U~ operand [64][NV]
-  static constexpr uint32_t OFF_BAR = OFF_UT + 64 * kRowB;
-  static constexpr uint32_t kSmem = OFF_BAR + 128;
+  static constexpr uint32_t OFF_OUT = OFF_UT + 64 * kRowB;       // bf16 output tile [64][NV], staged for the tile store
+  static constexpr uint32_t kSmem = OFF_OUT + 64 * kRowB;
+  static constexpr uint32_t OFF_BAR = OFF_SC + 768;              // barriers live in the unused tail of stage 0
+  static_assert(kStageB - OFF_BAR >= (2 * S_ + 2) * 8 + 16, "room for the barriers");
   static constexpr uint32_t kTmemCols = 2 * NV < 32 ? 32 : 2 * NV;
 };
 
@@ -120,6 +122,8 @@ __device__ __forceinline__ void ld32f(uint32_t taddr, float (&v)[32]) {
 // named barriers (0 is __syncthreads)
 constexpr int BAR_H_READY = 1;   // all compute threads arrive, MMA warp syncs: bf16 h is in shared memory
 constexpr int BAR_U_READY = 2;   // the U~ writers (half of them) arrive, MMA warp syncs: U~ operand is in shared memory
+constexpr int BAR_O_FREE = 3;    // output threads: the previous tile store has read the staging tile
+constexpr int BAR_O_FULL = 4;    // output threads: the staging tile is written
 __device__ __forceinline__ void named_arrive(int id, int count) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
@@ -129,7 +133,7 @@ __device__ __forceinline__ void named_sync(int id, int count) {
 
 template <int NV, bool KDA, int S, int CG>
 __global__ void __launch_bounds__(chain_threads(CG), 1)
-tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
+tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_o, ChainParams p) {
   using Cfg = ChainCfg<NV, S>;
   constexpr int NSL = 128 / NV;
   constexpr int NVT = NV / CG;                           // value channels per compute thread
@@ -165,6 +169,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tmap(&map_k);
+    prefetch_tmap(&map_o);
   }
   if (warp == 0) tmem_alloc(tmem_slot, Cfg::kTmemCols);
   tc_fence_before_sync();
@@ -177,6 +182,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   if (p.epoch == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
   uint8_t* sH = sm + Cfg::OFF_H;
   uint8_t* sUt = sm + Cfg::OFF_UT;
+  uint8_t* sOut = sm + Cfg::OFF_OUT;
 
   if (warp == W_PROD) {
     // ------------------------------------------------------------ producer
@@ -316,8 +322,14 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
         named_arrive(BAR_U_READY, NCOMP / 2 + 32);
         HA_PROF(chain, 8 * c + 3);
       } else {                                           // output rows: o = scale (O_loc + Q~ h)  (op #6)
+        // A full chunk leaves as one tile store per 64-channel block from a swizzled staging tile (a thread
+        // holds one token row, so direct stores would touch 32 lines per instruction); the ragged last chunk
+        // of a sequence is stored row by row, since a tile store could not stop at the sequence's end.
+        // (32-channel slices keep the direct stores: four per thread, cheaper than the staging's two barriers.)
+        const bool tile_out = NV > 32 && L == kChunk;
         __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
                               ((size_t)(tok0 + c * kChunk + i) * p.HV + j) * 128 + (size_t)slice * NV + cg0;
+        if (tile_out) named_sync(BAR_O_FREE, NCOMP / 2);
 #pragma unroll
         for (int c0 = 0; c0 < NVT; c0 += 32) {
           float d[32];
@@ -325,7 +337,9 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
           if (c0 > 0) load_img32(stage + Cfg::OFF_O, i, cg0 + c0, pre);
 #pragma unroll
           for (int q = 0; q < 32; ++q) d[q] = p.scale * (pre[q] + d[q]);
-          if (i < L) {
+          if (tile_out) {
+            store_brow32<NV, 64>(sOut, i, cg0 + c0, d);
+          } else if (i < L) {
 #pragma unroll
             for (int q = 0; q < 32; q += 8) {
               uint4 w;
@@ -333,6 +347,17 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
               w.z = pack_bf16(d[q + 4], d[q + 5]); w.w = pack_bf16(d[q + 6], d[q + 7]);
               *reinterpret_cast<uint4*>(orow + c0 + q) = w;
             }
+          }
+        }
+        if (tile_out) {
+          fence_proxy_async_smem();
+          named_sync(BAR_O_FULL, NCOMP / 2);
+          if (tid == 64) {                               // the first output thread issues and waits for the reads
+#pragma unroll
+            for (int b = 0; b < (NV + 63) / 64; ++b)
+              tma_store_3d(&map_o, sOut + b * 8192, slice * NV + b * 64, j, tok0 + c * kChunk);
+            bulk_commit();
+            bulk_wait_read_all();
           }
         }
       }
@@ -372,6 +397,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
   // Concurrent mode: do not finish before the prep grid has (it has published its last chunk by now), so that
   // work queued behind this kernel is also behind the prep kernel.
   if (p.epoch != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (tid == 64) bulk_wait_all();                        // this thread's tile stores have landed
   tc_fence_before_sync();
   __syncthreads();
   if (threadIdx.x == 0) HA_PROF_GT(chain, 901);
@@ -379,7 +405,8 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, ChainParams p) {
 }
 
 template <int NV, bool KDA, int S, int CG>
-cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, int grid, bool dependent, cudaStream_t stream) {
+cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMap* mo, int grid, bool dependent,
+                   cudaStream_t stream) {
   auto kern = tc_chain_kernel<NV, KDA, S, CG>;
   constexpr int smem = ChainCfg<NV, S>::kSmem;
   static_assert(smem <= 227 * 1024, "shared memory budget");
@@ -401,22 +428,23 @@ cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, int grid, bool 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = dependent ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, kern, *mk, *cp);
+  return cudaLaunchKernelEx(&cfg, kern, *mk, *mo, *cp);
 }
 
 // Slices of 64 and 128 value channels are worked on by two column groups of compute warps.
 template <bool KDA>
-cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, int nv, int grid, bool dependent,
-                        cudaStream_t stream) {
-  if (nv == 32) return run_nv<32, KDA, 3, 1>(cp, mk, grid, dependent, stream);
-  if (nv == 64) return run_nv<64, KDA, 3, 2>(cp, mk, grid, dependent, stream);
-  return run_nv<128, KDA, 2, 2>(cp, mk, grid, dependent, stream);
+cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMap* mo, int nv, int grid,
+                        bool dependent, cudaStream_t stream) {
+  if (nv == 32) return run_nv<32, KDA, 3, 1>(cp, mk, mo, grid, dependent, stream);
+  if (nv == 64) return run_nv<64, KDA, 3, 2>(cp, mk, mo, grid, dependent, stream);
+  return run_nv<128, KDA, 2, 2>(cp, mk, mo, grid, dependent, stream);
 }
 
 }  // namespace
 
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
-                            const CUtensorMap& mk, int nv, int64_t epoch, bool dependent, cudaStream_t stream) {
+                            const CUtensorMap& mk, const CUtensorMap& mo, int nv, int64_t epoch, bool dependent,
+                            cudaStream_t stream) {
   ChainParams cp;
   cp.h0 = a.h0; cp.hT = a.hT; cp.o = a.o;
   cp.seq_tok0 = plan.seq_tok0; cp.seq_len = plan.seq_len; cp.seq_chunk0 = plan.seq_chunk0;
@@ -426,14 +454,14 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   cp.epoch = epoch;
   const int grid = p.N * p.HV * (128 / nv);
   if (grid == 0) return cudaSuccess;
-  return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, nv, grid, dependent, stream)
-                                : run_variant<false>(&cp, &mk, nv, grid, dependent, stream);
+  return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, &mo, nv, grid, dependent, stream)
+                                : run_variant<false>(&cp, &mk, &mo, nv, grid, dependent, stream);
 }
 
 // Attributes (and loading) of the chain kernel instance a launch will use; see configure_tc_prep.
 cudaError_t configure_tc_chain(const Problem& p, int nv) {
-  return p.variant == HA_LA_KDA ? run_variant<true>(nullptr, nullptr, nv, 0, false, nullptr)
-                                : run_variant<false>(nullptr, nullptr, nv, 0, false, nullptr);
+  return p.variant == HA_LA_KDA ? run_variant<true>(nullptr, nullptr, nullptr, nv, 0, false, nullptr)
+                                : run_variant<false>(nullptr, nullptr, nullptr, nv, 0, false, nullptr);
 }
 
 }  // namespace ha_la
