@@ -97,15 +97,17 @@ int64_t next_epoch() {
   return (int64_t)(((uint64_t)tag << 32) | g_calls.fetch_add(1));
 }
 
-// Slice width (value channels per chain CTA) and launch mode.  The chain kernel is bound by the latency of its
-// two MMA round trips per chunk, which grows with the slice width (about 0.9 / 1.23 / 1.7 us per chunk at 32 /
-// 64 / 128 channels on B200) and does not depend on the number of CTAs.  Each CTA needs an SM of its own, so
-// the kernel's time is about  max(longest sequence, all sequences / SMs)  in chunk-times when the lengths differ
-// (more CTAs than SMs are started longest sequence first and pack well), and whole rounds when they do not:
-// with few chains the narrow slice wins, with many a wider one may.
+// Slice width (value channels per chain CTA) and launch mode, from a cost model measured on B200.
+// Chain kernel: bound by the latency of its two MMA round trips per chunk, which grows with the slice width (about
+// 0.9 / 1.23 / 1.7 us per chunk at 32 / 64 / 128 channels) and does not depend on the number of CTAs.  Each CTA
+// needs an SM of its own, so the kernel's time is about  max(longest sequence, all sequences / SMs)  in chunk-times
+// when the lengths differ (more CTAs than SMs are started longest sequence first and pack well), and whole rounds
+// when they do not: with few chains the narrow slice wins, with many a wider one may.
+// Prep kernel: throughput-bound, about 3.45 (GDN) / 12.1 (KDA) SM-microseconds per (chunk, head).
+// Back to back the two times add.  Concurrently (allowed while the chain's CTAs leave at least half of the SMs to
+// the prep kernel) the call takes the longer of the chain and of the prep kernel on the remaining SMs, plus the
+// wait for the first chunks and some interference.
 // Only bounds are known on the host: max_len for the longest sequence, max_chunks for the total.
-// Concurrent mode when the CTAs leave at least half of the SMs to the prep kernel and the slice is the narrow
-// one (with 64-channel slices the overlap measured no gain over back-to-back kernels with 32-channel slices).
 struct TcPlan { int nv; bool concurrent; };
 
 TcPlan plan_tc(const Problem& p) {
@@ -115,29 +117,38 @@ TcPlan plan_tc(const Problem& p) {
   const double items = (double)p.max_chunks * p.HV;
   const int widths[3] = {32, 64, 128};
   const double per_chunk_us[3] = {0.90, 1.23, 1.70};
-  int nv = 32;
-  double best = 1e30;
+  const double prep_us = items * (p.variant == HA_LA_KDA ? 12.1 : 3.45) / sms;
   // sequences of about the same length (batch rows, or a packed batch whose longest is close to its average)
   // cannot be packed any better than in rounds of one CTA per SM
   const double avg_len = p.N > 0 ? (double)p.T_total / p.N : 0.0;
   const bool even = avg_len <= 0.0 || p.max_len < 1.5 * avg_len;
-  for (int w = 0; w < 3; ++w) {
-    const long long ctas = chains * (128 / widths[w]);
-    const double serial = longest * per_chunk_us[w];
-    double est = serial;
-    if (ctas > sms) {
-      const double spread = 1.15 * items * (128 / widths[w]) * per_chunk_us[w] / sms;
-      est = even ? serial * (double)((ctas + sms - 1) / sms) : (serial > spread ? serial : spread);
-    }
-    if (est < best) { best = est; nv = widths[w]; }
-  }
+  bool may_overlap = !g_timer && p.max_chunks > 1;       // (timing wants one kernel at a time)
+  if (const char* e = getenv("HA_LA_TC_OVERLAP")) may_overlap = may_overlap && e[0] != '0';
+  int forced_nv = 0;
   if (const char* e = getenv("HA_LA_TC_NV")) {
     const int v = atoi(e);
-    if (v == 32 || v == 64 || v == 128) nv = v;
+    if (v == 32 || v == 64 || v == 128) forced_nv = v;
   }
-  bool conc = !g_timer && p.max_chunks > 1 && nv == 32 && chains * 4 * 2 <= sms;   // (timing wants one kernel at a time)
-  if (const char* e = getenv("HA_LA_TC_OVERLAP")) conc = conc && e[0] != '0';
-  return TcPlan{nv, conc};
+  TcPlan plan{32, false};
+  double best = 1e30;
+  for (int w = 0; w < 3; ++w) {
+    if (forced_nv && widths[w] != forced_nv) continue;
+    const long long ctas = chains * (128 / widths[w]);
+    const double serial = longest * per_chunk_us[w];
+    double chain_us = serial;
+    if (ctas > sms) {
+      const double spread = 1.15 * items * (128 / widths[w]) * per_chunk_us[w] / sms;
+      chain_us = even ? serial * (double)((ctas + sms - 1) / sms) : (serial > spread ? serial : spread);
+    }
+    const double back_to_back = prep_us + chain_us;
+    if (back_to_back < best) { best = back_to_back; plan = TcPlan{widths[w], false}; }
+    if (may_overlap && ctas * 2 <= sms) {
+      const double prep_beside = prep_us * sms / (double)(sms - ctas);
+      const double overlapped = 1.1 * (chain_us > prep_beside ? chain_us : prep_beside) + 12.0;
+      if (overlapped < best) { best = overlapped; plan = TcPlan{widths[w], true}; }
+    }
+  }
+  return plan;
 }
 
 }  // namespace
