@@ -11,6 +11,7 @@
 //   MMA1  D1[128 x NV] = [W ; Q~] h          rows 0..63: W h, rows 64..127: Q~ h      (M = 128)
 //         threads 0..63  : U~_i = (U_i - (W h)_i) e^{G_L - G_i}  -> bf16 operand in shared memory
 //         threads 64..127: o_i  = scale (O_loc,i + (Q~ h)_i)     -> global memory (op #6, uses the OLD state)
+//                          (64- and 128-channel slices: through a swizzled tile and a TMA tile store)
 //   MMA2  D2[128 x NV] = K^T U~              (A = the raw K tile, feature-major, by TMA)
 //         all threads    : h <- e^{G_L} h + D2                   (op #5 update, in place)
 //
