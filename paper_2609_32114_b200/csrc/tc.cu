@@ -103,10 +103,12 @@ int64_t next_epoch() {
 // needs an SM of its own, so the kernel's time is about  max(longest sequence, all sequences / SMs)  in chunk-times
 // when the lengths differ (more CTAs than SMs are started longest sequence first and pack well), and whole rounds
 // when they do not: with few chains the narrow slice wins, with many a wider one may.
-// Prep kernel: throughput-bound, about 3.45 (GDN) / 12.1 (KDA) SM-microseconds per (chunk, head).
+// Prep kernel: throughput-bound, about 3.45 (GDN) / 12.1 (KDA) SM-microseconds per (chunk, head), and never
+// faster than its rounds of one item per work group (3 per SM for GDN, 1 for KDA) at 9 / 12.5 us per item.
 // Back to back the two times add.  Concurrently (allowed while the chain's CTAs leave at least half of the SMs to
-// the prep kernel) the call takes the longer of the chain and of the prep kernel on the remaining SMs, plus the
-// wait for the first chunks and some interference.
+// the prep kernel) the call takes the longer of the chain and of the prep kernel on the remaining SMs (plus some
+// interference), plus the wait for the first chunks; with several sequences the prep kernel works through them
+// one after the other, so the last sequence's chain starts only when most of the prep work is done.
 // Only bounds are known on the host: max_len for the longest sequence, max_chunks for the total.
 struct TcPlan { int nv; bool concurrent; };
 
@@ -117,13 +119,24 @@ TcPlan plan_tc(const Problem& p) {
   const double items = (double)p.max_chunks * p.HV;
   const int widths[3] = {32, 64, 128};
   const double per_chunk_us[3] = {0.90, 1.23, 1.70};
-  const double prep_us = items * (p.variant == HA_LA_KDA ? 12.1 : 3.45) / sms;
+  const bool kda = p.variant == HA_LA_KDA;
+  auto prep_time = [&](int on_sms) {                     // the prep kernel on `on_sms` SMs
+    const double thru = items * (kda ? 12.1 : 3.45) / on_sms;
+    const double groups = (double)on_sms * (kda ? 1 : 3);
+    const double rounds = (double)(long long)((items + groups - 1) / groups) * (kda ? 12.5 : 9.0);
+    return thru > rounds ? thru : rounds;
+  };
+  const double prep_us = prep_time(sms);
   // sequences of about the same length (batch rows, or a packed batch whose longest is close to its average)
   // cannot be packed any better than in rounds of one CTA per SM
   const double avg_len = p.N > 0 ? (double)p.T_total / p.N : 0.0;
   const bool even = avg_len <= 0.0 || p.max_len < 1.5 * avg_len;
   bool may_overlap = !g_timer && p.max_chunks > 1;       // (timing wants one kernel at a time)
-  if (const char* e = getenv("HA_LA_TC_OVERLAP")) may_overlap = may_overlap && e[0] != '0';
+  bool force_overlap = false;                            // "2": side by side whenever that is legal (tests)
+  if (const char* e = getenv("HA_LA_TC_OVERLAP")) {
+    may_overlap = may_overlap && e[0] != '0';
+    force_overlap = may_overlap && e[0] == '2';
+  }
   int forced_nv = 0;
   if (const char* e = getenv("HA_LA_TC_NV")) {
     const int v = atoi(e);
@@ -140,11 +153,15 @@ TcPlan plan_tc(const Problem& p) {
       const double spread = 1.15 * items * (128 / widths[w]) * per_chunk_us[w] / sms;
       chain_us = even ? serial * (double)((ctas + sms - 1) / sms) : (serial > spread ? serial : spread);
     }
-    const double back_to_back = prep_us + chain_us;
+    const double back_to_back = prep_us + chain_us + (force_overlap ? 1e9 : 0.0);
     if (back_to_back < best) { best = back_to_back; plan = TcPlan{widths[w], false}; }
     if (may_overlap && ctas * 2 <= sms) {
-      const double prep_beside = prep_us * sms / (double)(sms - ctas);
-      const double overlapped = 1.1 * (chain_us > prep_beside ? chain_us : prep_beside) + 12.0;
+      const double prep_beside = 1.1 * prep_time(sms - (int)ctas);
+      double overlapped = (chain_us > prep_beside ? chain_us : prep_beside) + 12.0;
+      if (p.N > 1) {
+        const double last = prep_beside * (1.0 - 1.0 / p.N) + chain_us + 12.0;
+        if (last > overlapped) overlapped = last;
+      }
       if (overlapped < best) { best = overlapped; plan = TcPlan{widths[w], true}; }
     }
   }

@@ -158,34 +158,40 @@ def test_full_size_sampled(name, heads):
     print(name, res)
 
 
+@pytest.mark.parametrize("variant", ["gdn", "kda"])
 @pytest.mark.parametrize("nv", [32, 64, 128])
-def test_tc_every_slice_width(nv, monkeypatch):
-    """The tensor-core chain kernel at each value-slice width (normally chosen from the launch size)."""
+def test_tc_every_slice_width(nv, variant, monkeypatch):
+    """The tensor-core chain kernel at each value-slice width (normally chosen from the launch size): full
+    chunks (stored as tiles by the wider slices) and ragged last chunks (stored row by row) in one batch."""
     import paper_2609_32114_b200 as ha
 
     monkeypatch.setenv("HA_LA_TC_NV", str(nv))
-    w = synth.shrink(W["gdn_varlen"], seq_lens=[130, 700, 64], hk=2, hv=4, gate_shift=-1.0)
+    base = W["gdn_varlen"] if variant == "gdn" else W["kda_8k"]
+    w = synth.shrink(base, seq_lens=[130, 700, 64], hk=2, hv=4, gate_shift=-1.0, varlen=True)
     inp = synth.make_inputs(w, seed=31 + nv)
-    a = ha.make_args(variant="gdn", dtype="bf16", batch=1, seqlen=inp["T"], hk=2, hv=4, dk=128, dv=128, num_seqs=3)
+    a = ha.make_args(variant=variant, dtype="bf16", batch=1, seqlen=inp["T"], hk=2, hv=4, dk=128, dv=128, num_seqs=3)
     assert ha.ha_la_prefill_path(a) == "tc"
     helpers.check_parity(inp)
 
 
-@pytest.mark.parametrize("case", ["gdn", "kda", "varlen"])
+@pytest.mark.parametrize("case", ["gdn", "kda", "varlen", "gdn_nv64", "kda_nv64"])
 def test_concurrent_prep_and_chain_mode(case, monkeypatch):
-    """Default mode when the chain CTAs need at most half of the SMs: the chain kernel runs next to the
-    persistent prep kernel and takes each chunk as soon as its flag is published.  HA_LA_TC_OVERLAP=0
-    forces the sequential mode.  Same results in both, bit for bit, call after call."""
-    if case == "gdn":
+    """Concurrent mode (chosen by the launch planner while the chain CTAs need at most half of the SMs; forced
+    here with HA_LA_TC_OVERLAP=2): the chain kernel runs next to the persistent prep kernel and takes each
+    chunk as soon as its flag is published.  HA_LA_TC_OVERLAP=0 forces the sequential mode.  Same results in
+    both, bit for bit, call after call."""
+    if case.startswith("gdn"):
         w = synth.shrink(W["gdn_layer_4k"], seq_lens=[2048], hk=4, hv=4)
-    elif case == "kda":
+    elif case.startswith("kda"):
         w = synth.shrink(W["kda_8k"], seq_lens=[1000], hk=2, hv=4)
     else:
         w = synth.shrink(W["gdn_varlen"], seq_lens=[700, 0, 65, 1500], hk=2, hv=2)
+    if case.endswith("nv64"):
+        monkeypatch.setenv("HA_LA_TC_NV", "64")
     inp = synth.make_inputs(w, seed=37)
     monkeypatch.setenv("HA_LA_TC_OVERLAP", "0")
     o_seq, h_seq, st_seq = helpers.run_gpu(inp)
-    monkeypatch.delenv("HA_LA_TC_OVERLAP")
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", "2")
     o_con, h_con, st_con = helpers.run_gpu(inp)
     o_con2, h_con2, _ = helpers.run_gpu(inp)
     assert st_seq == 0 and st_con == 0
@@ -195,12 +201,13 @@ def test_concurrent_prep_and_chain_mode(case, monkeypatch):
     helpers.check_parity(inp)
 
 
-def test_workspace_contents_do_not_matter():
+def test_workspace_contents_do_not_matter(monkeypatch):
     """The workspace is scratch: whatever it holds on entry (small integers, all ones, an earlier call's
     flags) must not change the result -- in particular not pass for a 'chunk is ready' flag."""
     import torch
     import paper_2609_32114_b200 as ha
 
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", "2")          # concurrent mode whatever the planner would choose
     w = synth.shrink(W["gdn_layer_4k"], seq_lens=[1500], hk=2, hv=4)
     inp = synth.make_inputs(w, seed=41)
     d = helpers.to_device(inp)
@@ -224,13 +231,14 @@ def test_workspace_contents_do_not_matter():
     assert torch.equal(o3, o0) and torch.equal(h3, h0)
 
 
-def test_back_to_back_calls_share_a_workspace():
+def test_back_to_back_calls_share_a_workspace(monkeypatch):
     """Many calls queued on one stream without synchronising in between, alternating between two problems
     of different shape that share one workspace (so every call sees the other's leftovers and the
     launch-mode switches between concurrent and sequential): results must equal the first call's."""
     import torch
     import paper_2609_32114_b200 as ha
 
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", "2")          # concurrent mode wherever the chain leaves SMs free
     wa = synth.shrink(W["gdn_layer_4k"], seq_lens=[1024], hk=2, hv=2)           # few chains: concurrent mode
     wb = synth.shrink(W["gdn_varlen"], seq_lens=[200, 0, 333, 64] * 10, hk=2, hv=4)   # 160 chains: sequential
     ia, ib = synth.make_inputs(wa, seed=43), synth.make_inputs(wb, seed=44)
@@ -262,12 +270,13 @@ def test_back_to_back_calls_share_a_workspace():
     helpers.check_parity(ib)
 
 
-def test_two_streams_in_flight():
+def test_two_streams_in_flight(monkeypatch):
     """Calls on two streams at once, each with its own workspace: the prep and chain kernels of the two
     calls compete for the SMs (together they want more than there are), nothing may deadlock or mix up."""
     import torch
     import paper_2609_32114_b200 as ha
 
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", "2")          # both calls in the concurrent mode
     w1 = synth.shrink(W["gdn_layer_4k"], seq_lens=[2048], hk=8, hv=8)
     w2 = synth.shrink(W["kda_8k"], seq_lens=[1024], hk=4, hv=8)
     i1, i2 = synth.make_inputs(w1, seed=51), synth.make_inputs(w2, seed=52)
