@@ -3,12 +3,13 @@
 // Both kernels go on the caller's stream; the chain kernel is launched as a programmatic dependent of the
 // prep kernel, so it may start once every prep CTA is running.  Two modes:
 //   sequential: the chain kernel sets itself up under the prep kernel's tail and then waits for that whole grid;
-//   concurrent: when the chain CTAs need at most half of the SMs, the prep kernel is sized to the other SMs
+//   concurrent: when the chain CTAs need at most half of the SMs and the cost model below expects a gain, the
+//     prep kernel is sized to the other SMs
 //     (one CTA per SM) and the chain kernel consumes each chunk as soon as the prep work group of that chunk
 //     has published it (release/acquire flag per chunk in the workspace, stamped with a per-call epoch so that
 //     nothing has to be cleared).  The flags' producer is running (or done) before a consumer starts, whatever
 //     else the GPU is doing, so the consumer's bounded waits cannot starve.
-// HA_LA_TC_OVERLAP=0 forces the sequential mode.
+// HA_LA_TC_OVERLAP=0 forces the sequential mode, =2 the concurrent one wherever it is legal.
 #include <cuda.h>
 #include <stdlib.h>
 
