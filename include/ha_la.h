@@ -113,6 +113,16 @@ const char* ha_la_prefill_path(const ha_la_prefill_args* args);
 /* Number of kernels ha_la_prefill launches for these shapes (0 if unsupported).  Host only. */
 int ha_la_prefill_num_launches(const ha_la_prefill_args* args);
 
+/* How ha_la_prefill would launch the tensor-core kernels for these shapes (host only; pointers are
+ * ignored).  *slice_width = value channels per CTA of the sequential (state-passing) kernel: 32, 64 or
+ * 128 -- the "Computation Splitting" paragraph of Section 4: a head's state split into column sub-heads --
+ * or 0 on the CUDA-core path; *concurrent = 1 if that kernel runs beside the chunk-local kernel and
+ * takes each chunk as it is published, 0 if the two run back to back.  The choice comes from measured
+ * per-chunk costs of the two kernels and the bounds in `args` (sequences, longest sequence, total
+ * tokens); the environment switches HA_LA_TC_NV and HA_LA_TC_OVERLAP override it.
+ * Returns HA_LA_OK, or an error for invalid / unsupported shapes or NULL outputs.               */
+int ha_la_prefill_launch_plan(const ha_la_prefill_args* args, int* slice_width, int* concurrent);
+
 /* Profiling aid (the paper's "Metrics" paragraph times kernels with device events): the same work
  * as ha_la_prefill, with a CUDA event recorded on `cuda_stream` before every kernel and after the
  * last one.  Unlike ha_la_prefill it BLOCKS until the stream has drained, then writes the device

@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     ha_la_decode_raw,
     ha_la_prefill,
     ha_la_prefill_args,
+    ha_la_prefill_launch_plan,
     ha_la_prefill_num_launches,
     ha_la_prefill_path,
     ha_la_prefill_noalloc,

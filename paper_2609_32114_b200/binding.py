@@ -7,7 +7,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from typing import Optional
+from typing import Optional, Tuple
 
 HA_LA_GDN, HA_LA_KDA = 0, 1
 HA_LA_BF16, HA_LA_FP32 = 0, 1
@@ -31,6 +31,7 @@ EXPORTS = (
     "ha_la_prefill_noalloc_scratch_bytes",
     "ha_la_prefill_path",
     "ha_la_prefill_num_launches",
+    "ha_la_prefill_launch_plan",
     "ha_la_decode",
     "ha_la_status_string",
     "ha_la_version",
@@ -123,6 +124,8 @@ def load_library(path: Optional[str] = None):
     lib.ha_la_prefill_path.restype = ctypes.c_char_p
     lib.ha_la_prefill_num_launches.argtypes = [A]
     lib.ha_la_prefill_num_launches.restype = ctypes.c_int
+    lib.ha_la_prefill_launch_plan.argtypes = [A, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
+    lib.ha_la_prefill_launch_plan.restype = ctypes.c_int
     lib.ha_la_decode.argtypes = [ctypes.POINTER(ha_la_decode_args), ctypes.c_void_p]
     lib.ha_la_decode.restype = ctypes.c_int
     lib.ha_la_status_string.argtypes = [ctypes.c_int]
@@ -169,6 +172,15 @@ def ha_la_prefill_path(args: ha_la_prefill_args) -> Optional[str]:
 
 def ha_la_prefill_num_launches(args: ha_la_prefill_args) -> int:
     return load_library().ha_la_prefill_num_launches(ctypes.byref(args))
+
+
+def ha_la_prefill_launch_plan(args: ha_la_prefill_args) -> Tuple[int, bool]:
+    """(slice width of the sequential kernel or 0 on the CUDA-core path, kernels side by side?)."""
+    nv, conc = ctypes.c_int(0), ctypes.c_int(0)
+    rc = load_library().ha_la_prefill_launch_plan(ctypes.byref(args), ctypes.byref(nv), ctypes.byref(conc))
+    if rc != HA_LA_OK:
+        raise HaLaError(rc, "ha_la_prefill_launch_plan")
+    return nv.value, bool(conc.value)
 
 
 def ha_la_prefill_raw(args: ha_la_prefill_args, stream: int = 0) -> int:

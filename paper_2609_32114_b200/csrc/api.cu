@@ -96,6 +96,17 @@ int ha_la_prefill_num_launches(const ha_la_prefill_args* args) {
   return (needs_plan(args, p) ? 1 : 0) + (use_tc(p) ? tc_num_launches(p) : 1);
 }
 
+int ha_la_prefill_launch_plan(const ha_la_prefill_args* args, int* slice_width, int* concurrent) {
+  Problem p;
+  const int rc = make_problem(args, &p);
+  if (rc != HA_LA_OK) return rc;
+  if (!slice_width || !concurrent) return HA_LA_ERR_INVALID_ARG;
+  *slice_width = 0;
+  *concurrent = 0;
+  if (use_tc(p)) tc_launch_plan(p, slice_width, concurrent);
+  return HA_LA_OK;
+}
+
 int ha_la_prefill(const ha_la_prefill_args* a, void* cuda_stream) {
   Problem p;
   int rc = make_problem(a, &p);

@@ -68,6 +68,7 @@ bool simt_supported(const Problem& p);
 bool tc_supported(const Problem& p);
 size_t tc_workspace_bytes(const Problem& p);
 int tc_num_launches(const Problem& p);
+void tc_launch_plan(const Problem& p, int* slice_width, int* concurrent);   // what launch_tc would choose
 cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView plan, void* tc_ws,
                       cudaStream_t stream);
 

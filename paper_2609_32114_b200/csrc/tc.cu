@@ -181,6 +181,12 @@ size_t tc_workspace_bytes(const Problem& p) {
 
 int tc_num_launches(const Problem&) { return 2; }
 
+void tc_launch_plan(const Problem& p, int* slice_width, int* concurrent) {
+  const TcPlan tp = plan_tc(p);
+  *slice_width = tp.nv;
+  *concurrent = tp.concurrent ? 1 : 0;
+}
+
 cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView plan, void* tc_ws, cudaStream_t stream) {
   const TcPlan tp = plan_tc(p);
   const int nv = tp.nv;

@@ -87,3 +87,34 @@ def test_prefill_rejects_bad_pointers_without_launching(lib):
 def test_missing_library_fails_loudly(tmp_path):
     with pytest.raises(FileNotFoundError):
         ha.load_library(str(tmp_path / "libha_la.so"))
+
+
+def test_launch_plan_for_the_benchmark_shapes(lib, monkeypatch):
+    """Host-side launch planning (slice width of the sequential kernel, kernels side by side or back to back)
+    for the five benchmark shapes on a 148-SM GPU (the count assumed when no GPU is present)."""
+    for var in ("HA_LA_TC_NV", "HA_LA_TC_OVERLAP", "HA_LA_FORCE_SIMT"):
+        monkeypatch.delenv(var, raising=False)
+    plan = ha.ha_la_prefill_launch_plan
+    # one 4096-token sequence, 16 heads: 64 narrow-slice CTAs beside the chunk-local kernel
+    assert plan(_args()) == (32, True)
+    # 16384 tokens, 32 V-heads: 128 narrow CTAs would leave no SMs; 64 CTAs of 64 channels run beside it
+    assert plan(_args(seqlen=16384, hv=32)) == (64, True)
+    # KDA, 8192 tokens, 32 heads: its chunk-local kernel is too slow on half of the SMs: back to back
+    assert plan(_args(variant="kda", seqlen=8192, hk=32, hv=32)) == (32, False)
+    # packed batch of 8 sequences (139,389 tokens, longest 30,933): more CTAs than SMs, 64-channel slices
+    assert plan(_args(seqlen=139389, num_seqs=8, max_seqlen=30933)) == (64, False)
+    # fp32 inputs take the CUDA-core kernel: nothing to plan
+    assert plan(_args(dtype="fp32", dk=64, dv=64, hk=1, hv=1, seqlen=256)) == (0, False)
+    # a single chunk cannot overlap anything; tiny problems stay back to back
+    assert plan(_args(seqlen=64))[1] is False
+    assert plan(_args(seqlen=512)) == (32, False)
+    # the switches override the planner
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", "0")
+    assert plan(_args()) == (32, False)
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", "2")
+    assert plan(_args(seqlen=512)) == (32, True)
+    monkeypatch.setenv("HA_LA_TC_NV", "128")
+    assert plan(_args())[0] == 128
+    with pytest.raises(ha.HaLaError):
+        plan(_args(dk=96))
+    assert lib.ha_la_prefill_launch_plan(ctypes.byref(_args()), None, None) == binding.HA_LA_ERR_INVALID_ARG
