@@ -495,12 +495,16 @@ def main():
     t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
     t_flop = alg_flops / (peaks["bf16_tflops"] * 1e12)
     path_s = ms_per_step / 1e3
+    nv_plan, conc_plan = ha.ha_la_prefill_launch_plan(sets[0][0])
+    launch_mode = ("fp32 CUDA-core kernel" if nv_plan == 0 else
+                   f"{nv_plan}-channel slices, prep and chain kernels " + ("side by side" if conc_plan else "back to back"))
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic.get((w.name, dom)),
                 "kernel_alg_bytes": dom_bytes, "peak_source": peaks["source"],
                 "kernel_ms": kernel_ms,      # each kernel alone (sequential launches with events in between)
-                "launch_mode": "sequential" if os.environ.get("HA_LA_TC_OVERLAP", "1")[:1] == "0" else
-                               "default (prep and chain kernels overlap when the chain leaves SMs free)",
+                # what the timed steps used (kernel_ms is always back to back, and then with the planner's
+                # back-to-back slice width, which may differ)
+                "launch_mode": launch_mode,
                 "path": {"bound": "hbm" if t_hbm >= t_flop else "tensor", "roofline_us": 1e6 * max(t_hbm, t_flop),
                          "measured_us": 1e6 * path_s, "frac": max(t_hbm, t_flop) / path_s,
                          "achieved_gbs": alg_bytes / path_s / 1e9, "achieved_tflops": alg_flops / path_s / 1e12,
