@@ -325,3 +325,15 @@ def test_many_sequences_more_ctas_than_sms(variant):
     inp = synth.make_inputs(w, seed=61)
     res = helpers.check_parity(inp, scale=0.5)
     print(variant, res)
+
+
+def test_more_sequences_than_the_ranking_limit():
+    """4,500 short sequences (0..130 tokens) in one packed batch: beyond 4,096 sequences the plan kernel leaves
+    the launch order as given; the chain kernel then has thousands of CTAs, most of them with one or two chunks."""
+    rng = np.random.default_rng(11)
+    lens = [int(x) for x in rng.integers(0, 131, size=4500)]
+    w = synth.shrink(W["gdn_varlen"], seq_lens=lens, hk=1, hv=1, h0_std=0.02, varlen=True)
+    inp = synth.make_inputs(w, seed=67)
+    pairs = [(n, 0) for n in sorted(set(range(0, 4500, 23)) | {1, 2, 4095, 4096, 4097, 4499, int(np.argmax(lens))})]
+    res = helpers.check_parity(inp, pairs=pairs)
+    print(res)
