@@ -337,7 +337,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // Warp 1 stages the per-token scalars of an item one item ahead: GDN, log-gate and beta with cp.async (two
   // tokens per lane), scanned at the top of that item; KDA, beta likewise and the 64 x 128 log-gate rows by
   // bulk copies straight into the gate matrix (512 contiguous bytes per token).
-  auto stage_gates = [&](int j_, int L_, int tok0_) {
+  auto stage_gates = [&](int j_, int L_, int tok0_, bool rows) {
     if (warp == 1) {
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
@@ -351,7 +351,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
     }
-    if (KDA && warp == 8) {                              // a helper warp: off the other warps' critical path
+    if (KDA && rows && warp == 8) {                      // a helper warp: off the other warps' critical path
       if (lane == 0) mbar_expect_tx(bar_g, (uint32_t)L_ * 512u);
       __syncwarp();
 #pragma unroll
@@ -366,19 +366,41 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
   };
+  // KDA, helper warps (8..15): where the next item is (one thread), its gate rows (warp 8), and the gate rows of
+  // the item after it into L2 (warp 9; 32 KiB from HBM take a while).
+  auto helper_geom = [&]() {
+    if (tid == kPrepThreads) {
+      int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
+      bool hn = cjl + vstride < p.total;
+      if (hn) { item_geom(cjl + vstride, jn, jqn, Ln, tok0n); hn = Ln > 0; }
+      sNext[0] = hn ? 1 : 0; sNext[1] = jn; sNext[2] = jqn; sNext[3] = Ln; sNext[4] = tok0n;
+    }
+  };
+  auto helper_fetch = [&]() {                            // (after helper_geom and a barrier or __syncwarp)
+    if (warp == 8 && sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4], true);
+    if (warp == 9) {
+      int j2 = 0, jq2 = 0, L2 = 0, t2 = 0;
+      if (lane == 0 && cjl + 2 * vstride < p.total) item_geom(cjl + 2 * vstride, j2, jq2, L2, t2);
+      j2 = __shfl_sync(0xffffffffu, j2, 0);
+      L2 = __shfl_sync(0xffffffffu, L2, 0);
+      t2 = __shfl_sync(0xffffffffu, t2, 0);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int t = lane + 32 * h;
+        if (t < L2) bulk_prefetch_l2(p.g + ((size_t)(t2 + t) * p.HV + j2) * 128, 512);
+      }
+    }
+  };
   if (have) {
     if (tid == 0) issue_tiles(jq, tok0);
-    stage_gates(j, L, tok0);
+    stage_gates(j, L, tok0, true);
   }
   while (have) {
   const size_t cj = (size_t)cjl;
   if constexpr (KDA) {
-    // The previous item's bulk stores must have read their shared-memory sources before anything is overwritten.
-    if (tid == 0) {
-      if (prev_cj >= 0) bulk_wait_read_all();
-      issue_v(j, tok0);
-      publish_prev();
-    }
+    // (The previous item's last two images may still be leaving shared memory: nothing down to the gate-scaled
+    // operand copies touches their room; the wait for them, and the V tiles that land there, come after that.)
+    if (tid == 0) publish_prev();
     bsync();
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
     float* sGc = reinterpret_cast<float*>(sm + OFF_G);
@@ -397,9 +419,6 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       if (tid < 4) sFall[tid] = 0;
-      // A and P start as zero (entries above the diagonal are never written)
-      for (int idx = tid; idx < 64 * LDH * 2 / 16; idx += NT) reinterpret_cast<uint4*>(sAh)[idx] = make_uint4(0, 0, 0, 0);
-      for (int idx = tid; idx < 512; idx += NT) reinterpret_cast<uint4*>(sm + OFF_P)[idx] = make_uint4(0, 0, 0, 0);
     }
     if (warp == 0) mbar_wait(bar_g, lph, abort_flag);    // the raw log-gate rows (staged during the previous item)
     bsync();
@@ -521,6 +540,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     PP(0);
     const bool anyfall = (sFall[0] | sFall[1] | sFall[2] | sFall[3]) != 0;
     if (tid == 0) {                        // block-row I: D_I[128 x 16 (I + 1)] = [all K+ / Q+ rows] (K-^(I))^T;
+      // The previous item's images have had the gate passes' time to leave: A, P and V go where they were.
+      if (prev_cj >= 0) bulk_wait_read_all();
+      issue_v(j, tok0);
       tc_fence_after_sync();               // only rows 32 I .. 32 I + 31 (K+_I, Q+_I) of D_I are used
 #pragma unroll
       for (int I = 0; I < 4; ++I) {
@@ -536,7 +558,21 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       umma_commit(bar_mma);
     }
-    if (!anyfall) rescale_pass(true);
+    if (tid < 128) sQt[tid] = sGc[63 * LDG + tid];       // the chunk's total decay, for the chain kernel's scalars
+    if (!anyfall) {
+      rescale_pass(true);
+      // That was the last use of the gate matrix (the scalars above are a copy), so the helper warps can fetch
+      // the next item's gate rows into it right away, while the other warps solve: a warp needs some 3 k cycles
+      // to issue its 64 row copies, which the whole group used to wait for at the top of the next item.
+      if (is_main) {
+        asm volatile("bar.arrive 9, %0;" ::"r"(kKdaThreads) : "memory");
+      } else {
+        asm volatile("bar.sync 9, %0;" ::"r"(kKdaThreads) : "memory");   // every warp is done with the matrix
+        helper_geom();
+        if (warp == 8) __syncwarp();
+        helper_fetch();
+      }
+    }
     if (is_main) {                                       // the helper warps are done with this item's arithmetic
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
     mph ^= 1;
@@ -552,16 +588,21 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const uint32_t col = I == 0 ? 0 : (I == 1 ? 16 : (I == 2 ? 48 : 96));
       const uint32_t tl = tmem + (static_cast<uint32_t>(I * 32) << 16) + col;
       const float bi = sBeta[i];
-      for (int cb = warp >> 2; cb <= I; cb += 2) {
-        uint32_t r[16];
-        tmem_ld16(tl + 16 * cb, r);
-        tmem_ld_wait();
+      for (int cb = warp >> 2; cb < 4; cb += 2) {        // (pieces right of the diagonal block are zero)
         float v[16];
+        if (cb <= I) {
+          uint32_t r[16];
+          tmem_ld16(tl + 16 * cb, r);
+          tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          const int jj = 16 * cb + c;
-          const bool keep = isq ? jj <= i : jj < i;      // only the diagonal piece (cb == I) has entries to drop
-          v[c] = keep ? __uint_as_float(r[c]) * (isq ? 1.f : bi) : 0.f;
+          for (int c = 0; c < 16; ++c) {
+            const int jj = 16 * cb + c;
+            const bool keep = isq ? jj <= i : jj < i;    // only the diagonal piece (cb == I) has entries to drop
+            v[c] = keep ? __uint_as_float(r[c]) * (isq ? 1.f : bi) : 0.f;
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) v[c] = 0.f;
         }
         if (!isq) {
           uint4* d = reinterpret_cast<uint4*>(sAh + i * LDH + 16 * cb);
@@ -638,9 +679,6 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       publish_prev();                                    // (its wait for the stores overlaps the tiles' arrival)
       mbar_wait(bar_load, lph, abort_flag);
       PP(3);
-      // the previous item's W / U images must have left before V lands on one and A is written over the other
-      if (prev_cj >= 0) bulk_wait_read_all();
-      issue_v(j, tok0);
       tc_fence_after_sync();
       const uint32_t id = idesc_bf16(128, 64, false, false);
       const uint32_t base = smem_u32(sm + OFF_KQ);
@@ -650,6 +688,10 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         umma_ss(tmem, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(a, 16, 1024, kSwizzle128B), id, ks > 0);
       }
       umma_commit(bar_mma);
+      // the previous item's last two images must have left before V lands on one and A is written over the other
+      // (after the barrier below); the wait runs under the MMAs
+      if (prev_cj >= 0) bulk_wait_read_all();
+      issue_v(j, tok0);
     }
     if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);  // one warp polls; the others sleep at the barrier
     mph ^= 1;
@@ -845,36 +887,23 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     float* sc = p.ws.sc + (size_t)cj * kScFloats;
     const int t = tid - 64;                              // 0..191
     if constexpr (KDA) {
-      sc[t] = t < 64 ? 1.f : ex2(reinterpret_cast<const float*>(sm + OFF_G)[63 * LDG + (t - 64)]);
+      sc[t] = t < 64 ? 1.f : ex2(reinterpret_cast<const float*>(sm + OFF_QT)[t - 64]);
     } else {
       const float gl = sG[63];
       sc[t] = t < 64 ? __expf(gl - sG[t]) : __expf(gl);
     }
   }
   }  // is_main
-  // KDA: the helper warps have been waiting here since the gate-dependent passes; the gate matrix was read for
-  // the last time just above and the next item's whereabouts are known: stage its gate rows and betas.
+  // KDA: the helper warps have been waiting here.  Normally they fetched the next item's gate rows right after the
+  // gate-dependent passes; if a diagonal block was evaluated again from the gate matrix, they do it now.  The
+  // barrier also hands the next item's whereabouts (a helper thread's work) to the other warps.
   if constexpr (KDA) {
-    if (tid == kPrepThreads) {                           // a helper thread works out where the next item is
-      int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
-      bool hn = cjl + vstride < p.total;
-      if (hn) { item_geom(cjl + vstride, jn, jqn, Ln, tok0n); hn = Ln > 0; }
-      sNext[0] = hn ? 1 : 0; sNext[1] = jn; sNext[2] = jqn; sNext[3] = Ln; sNext[4] = tok0n;
-    }
+    const int* fall = reinterpret_cast<const int*>(sm + OFF_FALL);
+    const bool late = (fall[0] | fall[1] | fall[2] | fall[3]) != 0;
+    if (late) helper_geom();
     bsync();
-    if (sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4]);
-    if (warp == 9) {                                     // another helper warp: the gate rows of the item after
-      int j2 = 0, jq2 = 0, L2 = 0, t2 = 0;               // the next one, into L2 (32 KiB from HBM take a while)
-      if (lane == 0 && cjl + 2 * vstride < p.total) item_geom(cjl + 2 * vstride, j2, jq2, L2, t2);
-      j2 = __shfl_sync(0xffffffffu, j2, 0);
-      L2 = __shfl_sync(0xffffffffu, L2, 0);
-      t2 = __shfl_sync(0xffffffffu, t2, 0);
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int t = lane + 32 * h;
-        if (t < L2) bulk_prefetch_l2(p.g + ((size_t)(t2 + t) * p.HV + j2) * 128, 512);
-      }
-    }
+    if (late && !is_main) helper_fetch();
+    if (sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4], false);   // (betas, by one of the other warps)
   }
   if (is_main) {
   if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
@@ -915,7 +944,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
     bulk_commit();
   }
-  if (!KDA && sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4]);   // (after the barrier: thread 0 wrote sNext)
+  if (!KDA && sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4], false);   // (after the barrier: thread 0 wrote sNext)
   }  // is_main
   const bool have_n = sNext[0] != 0;
   const int jn = sNext[1], jqn = sNext[2], Ln = sNext[3], tok0n = sNext[4];
