@@ -230,6 +230,11 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   constexpr int G = kGroups<KDA>;
   extern __shared__ __align__(1024) uint8_t smem_raw[];  // no static shared memory in this kernel: 1024-aligned
   constexpr int NT = KDA ? kKdaThreads : kPrepThreads;   // threads of a work group
+  // Where the Q~ and O_loc images are staged for their bulk stores.  GDN: over the W and U images (which must
+  // have left by then).  KDA: over the gate-scaled operand copies, dead once the first product is complete, so
+  // that the group does not wait for the W / U / K e^{G_L-G} images to be read (48 KiB, some 1.5 k cycles).
+  constexpr uint32_t OFF_QI = KDA ? OFF_KQP : OFF_WT;
+  constexpr uint32_t OFF_OI = KDA ? OFF_KQP + 16384 : OFF_UT;
   const int grp = threadIdx.x / NT;                      // work group of this thread
   uint8_t* sm = smem_raw + grp * kGroupSmem;
   auto gsync = [&]() {                                   // barrier of the 8 warps of a group that run every phase
@@ -306,12 +311,14 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       L_ = min(kChunk, p.T_row - cc_ * kChunk);
     }
   };
-  auto issue_tiles = [&](int jq_, int tok0_) {           // thread 0: K and Q tiles of one item
+  auto issue_tiles_kb = [&](int jq_, int tok0_, int kb) { // feature half kb of the K and Q tiles of one item
+    tma_load_3d(sm + OFF_KQ + kb * 16384, &map_k, bar_load, kb * 64, jq_, tok0_);
+    tma_load_3d(sm + OFF_KQ + kb * 16384 + 8192, &map_q, bar_load, kb * 64, jq_, tok0_);
+  };
+  auto issue_tiles = [&](int jq_, int tok0_) {           // one thread: K and Q tiles of one item
     mbar_expect_tx(bar_load, 4 * 8192);
-    for (int kb = 0; kb < 2; ++kb) {
-      tma_load_3d(sm + OFF_KQ + kb * 16384, &map_k, bar_load, kb * 64, jq_, tok0_);
-      tma_load_3d(sm + OFF_KQ + kb * 16384 + 8192, &map_q, bar_load, kb * 64, jq_, tok0_);
-    }
+    issue_tiles_kb(jq_, tok0_, 0);
+    issue_tiles_kb(jq_, tok0_, 1);
   };
   auto issue_v = [&](int j_, int tok0_) {                // thread 0: V tiles (their room is free later than K's)
     mbar_expect_tx(bar_v, 2 * 8192);
@@ -398,9 +405,14 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   while (have) {
   const size_t cj = (size_t)cjl;
   if constexpr (KDA) {
-    // (The previous item's last two images may still be leaving shared memory: nothing down to the gate-scaled
-    // operand copies touches their room; the wait for them, and the V tiles that land there, come after that.)
-    if (tid == 0) publish_prev();
+    // The previous item's W / U / K e^{G_L-G} images (its first group of bulk stores, issued long ago) have left
+    // shared memory: V lands on one, the rescaling pass rewrites another.  Its Q~ / O_loc images (second group)
+    // sit where the gate-scaled operand copies go, and are waited for just before those are written.
+    if (tid == 0) {
+      if (prev_cj >= 0) bulk_wait_read_1();
+      issue_v(j, tok0);
+      publish_prev();
+    }
     bsync();
     // ---- op #1 Gate, per key channel: G[i][c] = cumulative log-gate, kept times log2(e) for ex2
     float* sGc = reinterpret_cast<float*>(sm + OFF_G);
@@ -440,6 +452,8 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       for (int i = 0; i < 16; ++i) sGc[(16 * sc_q + i) * LDG + sc_c] += add;
     }
     mbar_wait(bar_load, lph, abort_flag);                // every thread reads the K / Q tiles below
+    // the previous item's Q~ / O_loc images have left the room of the operand copies written next
+    if (tid == 0 && prev_cj >= 0) bulk_wait_read_all();
     bsync();
     PP(4);
 
@@ -539,10 +553,9 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     };
     PP(0);
     const bool anyfall = (sFall[0] | sFall[1] | sFall[2] | sFall[3]) != 0;
-    if (tid == 0) {                        // block-row I: D_I[128 x 16 (I + 1)] = [all K+ / Q+ rows] (K-^(I))^T;
-      // The previous item's images have had the gate passes' time to leave: A, P and V go where they were.
-      if (prev_cj >= 0) bulk_wait_read_all();
-      issue_v(j, tok0);
+    // The 32 MMAs of this step are issued by a thread of the last helper warp: issuing takes about as long as a
+    // warp's share of the rescaling pass below, and the other warps wait for the first eight, not for the helpers.
+    if (tid == kKdaThreads - 32) {         // block-row I: D_I[128 x 16 (I + 1)] = [all K+ / Q+ rows] (K-^(I))^T;
       tc_fence_after_sync();               // only rows 32 I .. 32 I + 31 (K+_I, Q+_I) of D_I are used
 #pragma unroll
       for (int I = 0; I < 4; ++I) {
@@ -567,6 +580,10 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (is_main) {
         asm volatile("bar.arrive 9, %0;" ::"r"(kKdaThreads) : "memory");
       } else {
+        // the helpers' part of the rescaled K / Q / K e^{G_L-G} tiles: visible to the tensor cores and the bulk
+        // stores (proxy fence) once the other warps have passed barrier 10, before the W / U products
+        fence_proxy_async_smem();
+        asm volatile("bar.arrive 10, %0;" ::"r"(kKdaThreads) : "memory");
         asm volatile("bar.sync 9, %0;" ::"r"(kKdaThreads) : "memory");   // every warp is done with the matrix
         helper_geom();
         if (warp == 8) __syncwarp();
@@ -806,6 +823,10 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       *reinterpret_cast<uint4*>(sm + OFF_TU + off) = pack8(tu);
     }
   }
+  if constexpr (KDA) {                                   // the helper warps' share of the rescaling pass is complete
+    const int* fall = reinterpret_cast<const int*>(sm + OFF_FALL);
+    if ((fall[0] | fall[1] | fall[2] | fall[3]) == 0) asm volatile("bar.sync 10, %0;" ::"r"(kKdaThreads) : "memory");
+  }
   fence_proxy_async_smem();
   tc_fence_before_sync();
   gsync();
@@ -883,6 +904,12 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if constexpr (KDA) bulk_store(p.ws.kd + (size_t)cj * kImgBytes, sm + OFF_KD, kImgBytes);
     bulk_commit();
   }
+  if (!KDA && tid == 32) {                               // where the next item is (idle thread, under the MMAs)
+    int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
+    bool hn = nxt < p.total;
+    if (hn) { item_geom(nxt, jn, jqn, Ln, tok0n); hn = Ln > 0; }
+    sNext[0] = hn ? 1 : 0; sNext[1] = jn; sNext[2] = jqn; sNext[3] = Ln; sNext[4] = tok0n;
+  }
   if (tid >= 64) {                                       // per-chunk scalars for the chain kernel
     float* sc = p.ws.sc + (size_t)cj * kScFloats;
     const int t = tid - 64;                              // 0..191
@@ -907,44 +934,42 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   }
   if (is_main) {
   if (warp == 0) mbar_wait(bar_mma, mph, abort_flag);
-  if (tid == 0) bulk_wait_read_all();                    // the W and U images were read; they receive the next two
+  // GDN: the W and U images must have been read, they receive the next two.  (KDA has room for those elsewhere.)
+  if (!KDA && tid == 0) bulk_wait_read_all();
   mph ^= 1;
   gsync();
   PP(12);
   tc_fence_after_sync();
   // Every MMA of this item is done, so the K / Q tile regions are free: start the next item's loads now
   // (its V tiles follow at the top of the loop, once the O_loc image has left their room).
-  if (tid == 0) {
-    if constexpr (KDA) {                                 // (a helper thread has worked out where the next item is)
-      if (sNext[0]) issue_tiles(sNext[2], sNext[4]);
-    } else {                                             // one thread works out where the next item is
-      int jn = 0, jqn = 0, Ln = 0, tok0n = 0;
-      bool hn = nxt < p.total;
-      if (hn) { item_geom(nxt, jn, jqn, Ln, tok0n); hn = Ln > 0; }
-      PP(14);
-      if (hn) issue_tiles(jqn, tok0n);
-      PP(15);
-      sNext[0] = hn ? 1 : 0; sNext[1] = jn; sNext[2] = jqn; sNext[3] = Ln; sNext[4] = tok0n;
+  // (Where the next item is was worked out meanwhile: KDA, by a helper thread; GDN, by thread 32 under the MMAs.
+  // Two threads of different warps share the four tile loads, so that no warp starts the epilogue much later.)
+  if (sNext[0]) {
+    if (tid == 0) {
+      mbar_expect_tx(bar_load, 4 * 8192);
+      issue_tiles_kb(sNext[2], sNext[4], 0);
+    } else if (tid == 32) {
+      issue_tiles_kb(sNext[2], sNext[4], 1);
     }
   }
   {
     // Q~^T and O_loc^T are complete in the accumulators; their images go where W^T and U^T were.
     float v[32];
     ld32(my_tmem, v);
-    store_half_row(v, rowq, hf, sm + OFF_WT);
+    store_half_row(v, rowq, hf, sm + OFF_QI);
     ld32(my_tmem + 64, v);
-    store_half_row(v, rowq, hf, sm + OFF_UT);
+    store_half_row(v, rowq, hf, sm + OFF_OI);
   }
   // The accumulators were read: the next item's first MMA may overwrite them after this barrier.
   fence_proxy_async_smem();
   tc_fence_before_sync();
   gsync();
   if (tid == 0) {
-    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_WT, kImgBytes);
-    bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
+    bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes + kImgBytes, sm + OFF_QI, kImgBytes);
+    bulk_store(p.ws.ol + (size_t)cj * kImgBytes, sm + OFF_OI, kImgBytes);
     bulk_commit();
   }
-  if (!KDA && sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4], false);   // (after the barrier: thread 0 wrote sNext)
+  if (!KDA && sNext[0]) stage_gates(sNext[1], sNext[3], sNext[4], false);   // (sNext: written before the barriers above)
   }  // is_main
   const bool have_n = sNext[0] != 0;
   const int jn = sNext[1], jqn = sNext[2], Ln = sNext[3], tok0n = sNext[4];
