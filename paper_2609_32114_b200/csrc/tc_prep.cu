@@ -553,21 +553,19 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     };
     PP(0);
     const bool anyfall = (sFall[0] | sFall[1] | sFall[2] | sFall[3]) != 0;
-    // The 32 MMAs of this step are issued by a thread of the last helper warp: issuing takes about as long as a
-    // warp's share of the rescaling pass below, and the other warps wait for the first eight, not for the helpers.
-    if (tid == kKdaThreads - 32) {         // block-row I: D_I[128 x 16 (I + 1)] = [all K+ / Q+ rows] (K-^(I))^T;
-      tc_fence_after_sync();               // only rows 32 I .. 32 I + 31 (K+_I, Q+_I) of D_I are used
+    // One product D[128 x 160] = [all K+ / Q+ rows] [K-^(0); K-^(1); K-^(2); K-^(3)]^T: the K- copies of the four
+    // block-rows are stacked (16 + 32 + 48 + 64 rows), so block-row I's result is rows 32 I .. 32 I + 31 (K+_I, Q+_I)
+    // of the columns where K-^(I) starts; the other row/column combinations are computed and never read (an MMA
+    // costs the same whatever its rows: eight instructions instead of one set of eight per block-row).
+    // Issued by a thread of the last helper warp, so that warp 0 starts its share of the rescaling pass at once.
+    if (tid == kKdaThreads - 32) {
+      tc_fence_after_sync();
+      const uint32_t id = idesc_bf16(128, 160, false, false);
 #pragma unroll
-      for (int I = 0; I < 4; ++I) {
-        const uint32_t id = idesc_bf16(128, 16 * (I + 1), false, false);
-        const uint32_t col = I == 0 ? 0 : (I == 1 ? 16 : (I == 2 ? 48 : 96));
-        const uint32_t r0 = col;                         // first K- row of this block-row = its column offset
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t a = smem_u32(sm + OFF_KQP) + (ks >> 2) * KQP_KB + (ks & 3) * 32;
-          const uint32_t bb = smem_u32(sm + OFF_KM) + (ks >> 2) * KM_KB + r0 * 128 + (ks & 3) * 32;
-          umma_ss(tmem + col, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(bb, 16, 1024, kSwizzle128B), id, ks > 0);
-        }
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t a = smem_u32(sm + OFF_KQP) + (ks >> 2) * KQP_KB + (ks & 3) * 32;
+        const uint32_t bb = smem_u32(sm + OFF_KM) + (ks >> 2) * KM_KB + (ks & 3) * 32;
+        umma_ss(tmem, smem_desc(a, 16, 1024, kSwizzle128B), smem_desc(bb, 16, 1024, kSwizzle128B), id, ks > 0);
       }
       umma_commit(bar_mma);
     }
@@ -831,6 +829,12 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   tc_fence_before_sync();
   gsync();
   PP(9);
+  if constexpr (KDA) {                                   // K e^{G_L-G} is complete (rescaling pass): its image leaves now,
+    if (tid == 0) {                                      // in a bulk group of its own, well ahead of the W / U images
+      bulk_store(p.ws.kd + (size_t)cj * kImgBytes, sm + OFF_KD, kImgBytes);
+      bulk_commit();
+    }
+  }
 
   // ---- op #4 W/U: W^T = K^T (T^W)^T, U^T = V^T (T^U)^T  (A operands feature-major straight from the TMA tiles)
   if (tid == 0) {
@@ -901,7 +905,6 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     bulk_store(p.ws.wq + (size_t)cj * 2 * kImgBytes, sm + OFF_WT, kImgBytes);
     bulk_commit();
     bulk_store(p.ws.u + (size_t)cj * kImgBytes, sm + OFF_UT, kImgBytes);
-    if constexpr (KDA) bulk_store(p.ws.kd + (size_t)cj * kImgBytes, sm + OFF_KD, kImgBytes);
     bulk_commit();
   }
   if (!KDA && tid == 32) {                               // where the next item is (idle thread, under the MMAs)
