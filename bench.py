@@ -487,7 +487,7 @@ def main():
     # (profiles/tc_prep_chain_gdn_layer_4k_ncu_full.md, profiles/tc_prep_chain_kda_8k_ncu_full.md,
     # profiles/tc_prep_chain_nv64_gdn_gva_16k_ncu_full.md); cold-cache replays
     ncu_traffic = {("gdn_layer_4k", "tc_chain"): 84.71e6 + 5.90e6, ("gdn_layer_4k", "tc_prep"): 50.92e6 + 15.08e6,
-                   ("kda_8k", "tc_prep"): 336.83e6 + 292.74e6, ("kda_8k", "tc_chain"): 338.74e6 + 56.45e6,
+                   ("kda_8k", "tc_prep"): 336.78e6 + 291.11e6, ("kda_8k", "tc_chain"): 338.73e6 + 56.62e6,
                    ("gdn_gva_16k", "tc_prep"): 272.71e6 + 487.64e6, ("gdn_gva_16k", "tc_chain"): 612.41e6 + 120.54e6}
     dom_bytes = kernel_alg_bytes.get(dom, alg_bytes)
     dom_s = kernel_ms[dom] / 1e3
