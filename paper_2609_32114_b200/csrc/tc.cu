@@ -100,7 +100,8 @@ int64_t next_epoch() {
 
 // Slice width (value channels per chain CTA) and launch mode, from a cost model measured on B200.
 // Chain kernel: bound by the latency of its two MMA round trips per chunk, which grows with the slice width (about
-// 0.9 / 1.23 / 1.7 us per chunk at 32 / 64 / 128 channels) and does not depend on the number of CTAs.  Each CTA
+// 0.9 / 1.23 / 1.5 us per chunk at 32 / 64 / 128 channels; the last is a kernel of its own that keeps the whole head's
+// state in tensor memory) and does not depend on the number of CTAs.  Each CTA
 // needs an SM of its own, so the kernel's time is about  max(longest sequence, all sequences / SMs)  in chunk-times
 // when the lengths differ (more CTAs than SMs are started longest sequence first and pack well), and whole rounds
 // when they do not: with few chains the narrow slice wins, with many a wider one may.
@@ -119,7 +120,7 @@ TcPlan plan_tc(const Problem& p) {
   const double longest = (double)((p.max_len + kChunk - 1) / kChunk);
   const double items = (double)p.max_chunks * p.HV;
   const int widths[3] = {32, 64, 128};
-  const double per_chunk_us[3] = {0.90, 1.23, 1.70};
+  const double per_chunk_us[3] = {0.90, 1.23, 1.50};
   const bool kda = p.variant == HA_LA_KDA;
   auto prep_time = [&](int on_sms) {                     // the prep kernel on `on_sms` SMs
     const double thru = items * (kda ? 10.2 : 3.45) / on_sms;

@@ -24,6 +24,7 @@
 // In the concurrent mode the producer warp also watches the prep kernel's per-chunk flags (32 at a time).
 // Every mbarrier wait and every flag wait is bounded.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "tc_common.cuh"
 #include "tc_ptx.cuh"
@@ -112,6 +113,16 @@ __device__ __forceinline__ void load_img32(const uint8_t* slice, int i, int c0, 
     v[q] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(base + sw128_offset(c0 + q, ch)));
 }
 
+// eight bf16 (16 bytes) -> fp32
+__device__ __forceinline__ void unpack8(const uint4& w, float (&f)[8]) {
+  const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(u[i] << 16);
+    f[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+  }
+}
+
 __device__ __forceinline__ void ld32f(uint32_t taddr, float (&v)[32]) {
   uint32_t r[32];
   tmem_ld32(taddr, r);
@@ -125,6 +136,7 @@ constexpr int BAR_H_READY = 1;   // all compute threads arrive, MMA warp syncs: 
 constexpr int BAR_U_READY = 2;   // the U~ writers (half of them) arrive, MMA warp syncs: U~ operand is in shared memory
 constexpr int BAR_O_FREE = 3;    // output threads: the previous tile store has read the staging tile
 constexpr int BAR_O_FULL = 4;    // output threads: the staging tile is written
+                                 // (the whole-head kernel has two tiles: ids 3, 4 for tile 0 and 5, 6 for tile 1)
 __device__ __forceinline__ void named_arrive(int id, int count) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
@@ -405,6 +417,335 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
   if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Whole-head variant: one CTA owns all 128 value channels of a (sequence, V-head) and keeps the state TRANSPOSED
+// in tensor memory: lane = value channel v, columns = key channels.  Both products of a chunk then take their
+// state-dependent operand from tensor memory (the A operand of tcgen05.mma may live there), and the operand images
+// of the workspace serve unchanged as B operands from shared memory:
+//   MMA1  D1^T[v][0:64 | 64:128] = h^T [W ; Q~]^T      A = h^T (bf16 pairs, tensor memory), B = the W / Q~ images
+//         U~^T[v][i] = (U^T[v][i] - D1^T[v][i]) e^{G_L - G_i}   -> bf16 pairs straight back into tensor memory
+//   MMA2  D2^T[v][k] = U~^T K~                          A = U~^T (tensor memory), B = the K tile (K e^{G_L-G}: KDA)
+//         h^T[v][k] <- gamma_k h^T[v][k] + D2^T[v][k]   fp32 in registers, bf16 pairs back into tensor memory
+//         o[i][v]   = scale (O_loc^T[v][i] + D1^T[v][64 + i])   (after the update, under the next chunk's MMA1:
+//                                                                D1 alternates between two accumulators)
+// No operand goes through shared memory, so the two proxy fences per chunk of the sliced kernel (and its operand
+// stores) are gone, and the twelve MMA instructions of a chunk serve 128 value channels instead of 32 or 64.
+// Measured: about 1.5 us per chunk (the MMAs with a tensor-memory A operand and a 128-wide B run at about half
+// of the tensor peak and are the limit), against 0.9 us on FOUR SMs for 32-channel slices: the cheapest way
+// through a chunk in SM-time, the slowest in latency.
+// Eight compute warps: warp w works on lanes 32 (w % 4).. and on half w / 4 of the columns of each accumulator;
+// two more warps copy the output rows from a shared-memory tile to global memory.
+constexpr int kTThreads = 384;                           // 8 compute warps + producer warp + MMA warp + 2 output warps
+
+struct ChainTCfg {
+  static constexpr int kStages = 2;
+  static constexpr uint32_t OFF_WQ = 0;                          // 32 KiB: W image, Q~ image
+  static constexpr uint32_t OFF_K = 32768;                       // 16 KiB  [kb][64 tok][64 feat]
+  static constexpr uint32_t OFF_U = 49152;                       // 16 KiB: U image
+  static constexpr uint32_t OFF_O = 65536;                       // 16 KiB: O_loc image
+  static constexpr uint32_t OFF_SC = 81920;                      // 192 floats
+  static constexpr uint32_t kStageB = 82944;
+  static constexpr uint32_t kTxBytes = 32768 + 16384 + 16384 + 16384 + 768;
+  static constexpr uint32_t OFF_BAR = OFF_SC + 768 + 128;        // barriers: in the unused tail of stage 0
+  static constexpr uint32_t OFF_OUT = kStages * kStageB;         // two bf16 output tiles [2 x 64 ch blocks][64 tok], swizzled
+  static constexpr uint32_t kSmem = OFF_OUT + 2 * 16384;
+  static constexpr uint32_t kTmemCols = 512;
+  static constexpr uint32_t TM_D1 = 0, TM_D2 = 256, TM_H = 384, TM_UT = 448;   // D1: two accumulators of 128
+};
+
+template <bool KDA>
+__global__ void __launch_bounds__(kTThreads, 1)
+tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_o, ChainParams p) {
+  using Cfg = ChainTCfg;
+  constexpr int S = Cfg::kStages;
+  constexpr int NCOMP = 256;
+  constexpr int W_PROD = 8, W_MMA = 9, W_OUT = 10;  // warps 10 and 11 write o
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* sm = smem_raw;
+  uint64_t* bar_full = reinterpret_cast<uint64_t*>(sm + Cfg::OFF_BAR);
+  uint64_t* bar_empty = bar_full + S;
+  uint64_t* bar_mma1 = bar_empty + S;
+  uint64_t* bar_mma2 = bar_mma1 + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mma2 + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const int lane = tid & 31;
+  const int nj = blockIdx.x;
+  const int j = nj % p.HV;
+  const int n = p.seq_order ? p.seq_order[nj / p.HV] : nj / p.HV;
+  const int jq = j / (p.HV / p.HK);
+  const int tok0 = p.seq_tok0 ? p.seq_tok0[n] : n * p.T_row;
+  const int len = p.seq_tok0 ? p.seq_len[n] : p.T_row;
+  const int chunk0 = p.seq_tok0 ? p.seq_chunk0[n] : n * p.cps;
+  const int nchunks = (len + kChunk - 1) / kChunk;
+
+  if (tid == 0) {
+    for (int i = 0; i < S; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], NCOMP); }
+    mbar_init(bar_mma1, 1);
+    mbar_init(bar_mma2, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tmap(&map_k);
+    prefetch_tmap(&map_o);
+  }
+  if (warp == 0) tmem_alloc(tmem_slot, Cfg::kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+  if (p.epoch == 0) asm volatile("griddepcontrol.wait;" ::: "memory");   // sequential mode: the prep grid is done
+
+  if (warp == W_PROD) {
+    // ------------------------------------------------------------ producer (as in the sliced kernel)
+    int ready_upto = p.epoch != 0 ? 0 : nchunks;
+    for (int c = 0; c < nchunks; ++c) {
+      if (c >= ready_upto) {
+        int got = 0;
+        for (uint32_t it = 0; it < kSpinLimit && !*abort_flag; ++it) {
+          const int cc = c + lane;
+          bool ok = false;
+          if (cc < nchunks)
+            ok = *reinterpret_cast<const volatile int64_t*>(p.ws.flags + (size_t)(chunk0 + cc) * p.HV + j) == p.epoch;
+          const unsigned m = __ballot_sync(0xffffffffu, ok);
+          got = __ffs(~m) - 1;
+          if (got < 0) got = 32;
+          if (got > 0) break;
+          __nanosleep(100);
+        }
+        if (got == 0) *abort_flag = 1;
+        ready_upto = c + (got > 0 ? got : nchunks);
+        __threadfence();
+        fence_proxy_async_all();
+      }
+      if (lane == 0) {
+        const int st = c % S;
+        if (c >= S) mbar_wait(&bar_empty[st], ((c / S) - 1) & 1, abort_flag);
+        uint8_t* stage = sm + st * Cfg::kStageB;
+        const size_t cj = (size_t)(chunk0 + c) * p.HV + j;
+        mbar_expect_tx(&bar_full[st], Cfg::kTxBytes);
+        bulk_load(stage + Cfg::OFF_WQ, p.ws.wq + cj * 2 * kImgBytes, 32768, &bar_full[st]);
+        if constexpr (KDA) {
+          bulk_load(stage + Cfg::OFF_K, p.ws.kd + cj * kImgBytes, 16384, &bar_full[st]);
+        } else {
+          tma_load_3d(stage + Cfg::OFF_K, &map_k, &bar_full[st], 0, jq, tok0 + c * kChunk);
+          tma_load_3d(stage + Cfg::OFF_K + 8192, &map_k, &bar_full[st], 64, jq, tok0 + c * kChunk);
+        }
+        bulk_load(stage + Cfg::OFF_U, p.ws.u + cj * kImgBytes, 16384, &bar_full[st]);
+        bulk_load(stage + Cfg::OFF_SC, p.ws.sc + cj * kScFloats, 768, &bar_full[st]);
+        bulk_load(stage + Cfg::OFF_O, p.ws.ol + cj * kImgBytes, 16384, &bar_full[st]);
+      }
+      __syncwarp();
+    }
+  } else if (warp == W_MMA) {
+    // ------------------------------------------------------------ MMA issue
+    // A from tensor memory (K-major by construction), B from shared memory, MN-major (the images are feature-
+    // major: rows = the K index of these products, 128 swizzled bytes of the N index each).
+    const uint32_t id = idesc_bf16(128, 128, false, true);
+    const bool lead = lane == 0;
+    for (int c = 0; c < nchunks; ++c) {
+      const int st = c % S;
+      const uint32_t stage = smem_u32(sm + st * Cfg::kStageB);
+      const uint64_t dWQ = smem_desc(stage + Cfg::OFF_WQ, 16384, 1024, kSwizzle128B);   // N = 64 W + 64 Q~ tokens
+      const uint64_t dK = smem_desc(stage + Cfg::OFF_K, 8192, 1024, kSwizzle128B);      // N = 2 x 64 key channels
+      const uint32_t d1 = tmem + Cfg::TM_D1 + (c & 1) * 128;
+      if (lead) mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
+      named_sync(BAR_H_READY, NCOMP + 32);               // h^T (bf16 pairs) of the previous chunk is in tensor memory
+      if (lead) {
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)                    // K = d_k: 16 key channels = 8 columns of A, 2048 B of B
+          umma_ts(d1, tmem + Cfg::TM_H + ks * 8, dWQ + ks * (2048u >> 4), id, ks > 0);
+        umma_commit(bar_mma1);
+      }
+      named_sync(BAR_U_READY, NCOMP + 32);               // U~^T is in tensor memory
+      if (lead) {
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)                    // K = tokens: 16 tokens = 8 columns of A, 2048 B of B
+          umma_ts(tmem + Cfg::TM_D2, tmem + Cfg::TM_UT + ks * 8, dK + ks * (2048u >> 4), id, ks > 0);
+        umma_commit(bar_mma2);
+      }
+    }
+  } else if (warp >= W_OUT) {
+    // ------------------------------------------------------------ output rows: the compute warps leave a chunk's o
+    // as a token-major tile in shared memory (two tiles, used alternately); these two warps copy it out with plain
+    // 16-byte loads and stores, two whole token rows (512 contiguous bytes) per store instruction.  Plain accesses
+    // on both sides: no proxy fence (which takes thousands of cycles in this kernel, with 80 KiB of bulk loads per
+    // chunk in flight), and no global stores on the compute warps (a warp there holds 32 channels of a token).
+    const int ht = tid - W_OUT * 32;                     // 0..63
+    named_arrive(BAR_O_FREE, NCOMP + 64);                // both tiles start out free
+    named_arrive(BAR_O_FREE + 2, NCOMP + 64);
+    for (int c = 0; c < nchunks; ++c) {
+      const int b = c & 1;
+      const int L = min(kChunk, len - c * kChunk);
+      named_sync(BAR_O_FULL + 2 * b, NCOMP + 64);
+      const uint8_t* tile = sm + Cfg::OFF_OUT + b * 16384;
+      __nv_bfloat16* obase = reinterpret_cast<__nv_bfloat16*>(p.o) + ((size_t)(tok0 + c * kChunk) * p.HV + j) * 128;
+      const int k = ht & 15;                             // 16-byte piece of a token row (8 channels)
+#pragma unroll 4
+      for (int it = 0; it < 16; ++it) {
+        const int t = it * 4 + (ht >> 4);
+        const uint4 w = *reinterpret_cast<const uint4*>(tile + (k >> 3) * 8192 + sw128_offset(t, k & 7));
+        if (t < L) *reinterpret_cast<uint4*>(obase + (size_t)t * p.HV * 128 + k * 8) = w;
+      }
+      named_arrive(BAR_O_FREE + 2 * b, NCOMP + 64);
+    }
+  } else {
+    // ------------------------------------------------------------ compute
+    const int v = (warp & 3) * 32 + lane;                // value channel = tensor-memory lane
+    const int g = warp >> 2;                             // which half of the columns
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    float h[64];                                         // h^T[v][64 g .. 64 g + 63]
+    {
+      const size_t base = ((size_t)n * p.HV + j) * 128 * 128 + v;
+#pragma unroll
+      for (int q = 0; q < 64; ++q) h[q] = p.h0 ? p.h0[base + (size_t)(64 * g + q) * 128] : 0.f;
+    }
+    auto store_h = [&]() {                               // bf16 pairs of this thread's 64 key channels -> A operand
+#pragma unroll
+      for (int c0 = 0; c0 < 64; c0 += 32) {
+        uint32_t r[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) r[q] = pack_bf16(h[c0 + 2 * q], h[c0 + 2 * q + 1]);
+        tmem_st16(tmem + Cfg::TM_H + lane_base + 32 * g + c0 / 2, r);
+      }
+      tmem_st_wait();
+    };
+    store_h();
+    tc_fence_before_sync();
+    named_arrive(BAR_H_READY, NCOMP + 32);
+
+    // o of chunk c: after the state update, while the tensor cores work on the next chunk
+    auto output_part = [&](int c) {
+      const int st = c % S;
+      const uint8_t* stage = sm + st * Cfg::kStageB;
+      const int L = min(kChunk, len - c * kChunk);
+      float d[32];
+      ld32f(tmem + Cfg::TM_D1 + (c & 1) * 128 + lane_base + 64 + 32 * g, d);
+      float ol[32];
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        unpack8(*reinterpret_cast<const uint4*>(stage + Cfg::OFF_O + sw128_offset(v, 4 * g + q)),
+                *reinterpret_cast<float(*)[8]>(ol + 8 * q));
+      mbar_arrive(&bar_empty[st]);                       // last read of the stage by this thread
+      // hand the 32 tokens of this thread's channel to the output warps (token-major tile, 2-byte stores: a warp
+      // writes 64 contiguous bytes of a token row per instruction)
+      uint8_t* tile = sm + Cfg::OFF_OUT + (c & 1) * 16384 + (v >> 6) * 8192 + (v & 7) * 2;
+      named_sync(BAR_O_FREE + 2 * (c & 1), NCOMP + 64);  // the output warps are done with this tile's last contents
+#pragma unroll
+      for (int q = 0; q < 32; ++q) {
+        const int t = 32 * g + q;
+        *reinterpret_cast<__nv_bfloat16*>(tile + sw128_offset(t, (v & 63) >> 3)) =
+            __float2bfloat16_rn(p.scale * (ol[q] + d[q]));
+      }
+      named_arrive(BAR_O_FULL + 2 * (c & 1), NCOMP + 64);
+    };
+
+    for (int c = 0; c < nchunks; ++c) {
+      const int st = c % S;
+      const uint8_t* stage = sm + st * Cfg::kStageB;
+      const uint32_t ph = c & 1;
+      HA_PROF(chain, 8 * c + 0);
+      mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
+      HA_PROF(chain, 8 * c + 1);
+      const float* sc = reinterpret_cast<const float*>(stage + Cfg::OFF_SC);
+      // U^T[v][32 g .. 32 g + 31], fetched while MMA1 runs
+      float u[32];
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        unpack8(*reinterpret_cast<const uint4*>(stage + Cfg::OFF_U + sw128_offset(v, 4 * g + q)),
+                *reinterpret_cast<float(*)[8]>(u + 8 * q));
+      mbar_wait(bar_mma1, ph, abort_flag);
+      HA_PROF(chain, 8 * c + 2);
+      tc_fence_after_sync();
+      {
+        float d[32];
+        ld32f(tmem + Cfg::TM_D1 + (c & 1) * 128 + lane_base + 32 * g, d);
+        uint32_t r[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          const float2 dc = *reinterpret_cast<const float2*>(sc + 32 * g + 2 * q);   // e^{G_L - G_i}, two tokens
+          r[q] = pack_bf16((u[2 * q] - d[2 * q]) * dc.x, (u[2 * q + 1] - d[2 * q + 1]) * dc.y);
+        }
+        tmem_st16(tmem + Cfg::TM_UT + lane_base + 16 * g, r);
+        tmem_st_wait();
+      }
+      tc_fence_before_sync();
+      named_arrive(BAR_U_READY, NCOMP + 32);
+      HA_PROF(chain, 8 * c + 3);
+
+      mbar_wait(bar_mma2, ph, abort_flag);
+      HA_PROF(chain, 8 * c + 4);
+      tc_fence_after_sync();
+#pragma unroll
+      for (int c0 = 0; c0 < 64; c0 += 32) {
+        float d[32];
+        ld32f(tmem + Cfg::TM_D2 + lane_base + 64 * g + c0, d);
+        if constexpr (KDA) {
+#pragma unroll
+          for (int q = 0; q < 32; q += 4) {
+            const float4 gm = *reinterpret_cast<const float4*>(sc + 64 + 64 * g + c0 + q);   // decay per key channel
+            h[c0 + q] = fmaf(gm.x, h[c0 + q], d[q]);
+            h[c0 + q + 1] = fmaf(gm.y, h[c0 + q + 1], d[q + 1]);
+            h[c0 + q + 2] = fmaf(gm.z, h[c0 + q + 2], d[q + 2]);
+            h[c0 + q + 3] = fmaf(gm.w, h[c0 + q + 3], d[q + 3]);
+          }
+        } else {
+          const float gm = sc[64];                         // one decay for the whole chunk
+#pragma unroll
+          for (int q = 0; q < 32; ++q) h[c0 + q] = fmaf(gm, h[c0 + q], d[q]);
+        }
+      }
+      store_h();
+      tc_fence_before_sync();
+      named_arrive(BAR_H_READY, NCOMP + 32);
+      HA_PROF(chain, 8 * c + 5);
+      output_part(c);
+      HA_PROF(chain, 8 * c + 6);
+    }
+
+    if (p.hT) {
+      const size_t base = ((size_t)n * p.HV + j) * 128 * 128 + v;
+#pragma unroll
+      for (int q = 0; q < 64; ++q) p.hT[base + (size_t)(64 * g + q) * 128] = h[q];
+    }
+  }
+
+  if (warp == W_MMA) named_sync(BAR_H_READY, NCOMP + 32);  // pairs with the compute warps' last arrival
+  if (*abort_flag && tid == 0) report_status(p.status, HA_LA_ERR_TIMEOUT);
+  if (p.epoch != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
+}
+
+template <bool KDA>
+cudaError_t run_t(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMap* mo, int grid, bool dependent,
+                  cudaStream_t stream) {
+  auto kern = tc_chain_t_kernel<KDA>;
+  constexpr int smem = ChainTCfg::kSmem;
+  static_assert(smem <= 227 * 1024, "shared memory budget");
+  if (!cp) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  }
+  timer_mark(stream, "tc_chain");
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kTThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, *mk, *mo, *cp);
+}
+
 template <int NV, bool KDA, int S, int CG>
 cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMap* mo, int grid, bool dependent,
                    cudaStream_t stream) {
@@ -438,7 +779,10 @@ cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, const CUte
                         bool dependent, cudaStream_t stream) {
   if (nv == 32) return run_nv<32, KDA, 3, 1>(cp, mk, mo, grid, dependent, stream);
   if (nv == 64) return run_nv<64, KDA, 3, 2>(cp, mk, mo, grid, dependent, stream);
-  return run_nv<128, KDA, 2, 2>(cp, mk, mo, grid, dependent, stream);
+  if (const char* e = getenv("HA_LA_TC_WIDE_SLICED")) {
+    if (e[0] == '1') return run_nv<128, KDA, 2, 2>(cp, mk, mo, grid, dependent, stream);
+  }
+  return run_t<KDA>(cp, mk, mo, grid, dependent, stream);
 }
 
 }  // namespace
