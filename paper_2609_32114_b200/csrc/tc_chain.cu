@@ -773,16 +773,13 @@ cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, const CUtensorM
   return cudaLaunchKernelEx(&cfg, kern, *mk, *mo, *cp);
 }
 
-// Slices of 64 and 128 value channels are worked on by two column groups of compute warps.
+// Slices of 64 value channels are worked on by two column groups of compute warps.
 template <bool KDA>
 cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMap* mo, int nv, int grid,
                         bool dependent, cudaStream_t stream) {
   if (nv == 32) return run_nv<32, KDA, 3, 1>(cp, mk, mo, grid, dependent, stream);
   if (nv == 64) return run_nv<64, KDA, 3, 2>(cp, mk, mo, grid, dependent, stream);
-  if (const char* e = getenv("HA_LA_TC_WIDE_SLICED")) {
-    if (e[0] == '1') return run_nv<128, KDA, 2, 2>(cp, mk, mo, grid, dependent, stream);
-  }
-  return run_t<KDA>(cp, mk, mo, grid, dependent, stream);
+  return run_t<KDA>(cp, mk, mo, grid, dependent, stream);      // all 128 channels: the whole-head kernel
 }
 
 }  // namespace
