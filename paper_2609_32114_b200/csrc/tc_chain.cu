@@ -435,7 +435,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
 // through a chunk in SM-time, the slowest in latency.
 // Eight compute warps: warp w works on lanes 32 (w % 4).. and on half w / 4 of the columns of each accumulator;
 // two more warps copy the output rows from a shared-memory tile to global memory.
-constexpr int kTThreads = 384;                           // 8 compute warps + producer warp + MMA warp + 2 output warps
+constexpr int t_threads(int cg) { return (4 * cg + 4) * 32; }   // compute warps + producer, MMA and 2 output warps
 
 struct ChainTCfg {
   static constexpr int kStages = 2;
@@ -453,13 +453,16 @@ struct ChainTCfg {
   static constexpr uint32_t TM_D1 = 0, TM_D2 = 256, TM_H = 384, TM_UT = 448;   // D1: two accumulators of 128
 };
 
-template <bool KDA>
-__global__ void __launch_bounds__(kTThreads, 1)
+template <bool KDA, int CG>
+__global__ void __launch_bounds__(t_threads(CG), 1)
 tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_o, ChainParams p) {
   using Cfg = ChainTCfg;
   constexpr int S = Cfg::kStages;
-  constexpr int NCOMP = 256;
-  constexpr int W_PROD = 8, W_MMA = 9, W_OUT = 10;  // warps 10 and 11 write o
+  constexpr int NCOMP = 128 * CG;                        // compute threads: CG column groups of four warps
+  constexpr int TOK = 64 / CG;                           // tokens per thread in the U~ and output epilogues
+  constexpr int KC = 128 / CG;                           // key channels per thread in the state update
+  constexpr int W_PROD = 4 * CG, W_MMA = 4 * CG + 1, W_OUT = 4 * CG + 2;   // the last two warps write o
+  static_assert(CG == 2 || CG == 4, "two or four column groups");
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* sm = smem_raw;
   uint64_t* bar_full = reinterpret_cast<uint64_t*>(sm + Cfg::OFF_BAR);
@@ -595,21 +598,38 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   } else {
     // ------------------------------------------------------------ compute
     const int v = (warp & 3) * 32 + lane;                // value channel = tensor-memory lane
-    const int g = warp >> 2;                             // which half of the columns
+    const int g = warp >> 2;                             // column group
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    float h[64];                                         // h^T[v][64 g .. 64 g + 63]
+    auto ld_cols = [&](uint32_t taddr, float (&d)[TOK]) {     // TOK consecutive fp32 columns of this lane
+      if constexpr (TOK == 32) {
+        ld32f(taddr, d);
+      } else {
+        uint32_t r[16];
+        tmem_ld16(taddr, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int q = 0; q < 16; ++q) d[q] = __uint_as_float(r[q]);
+      }
+    };
+    auto img_row = [&](const uint8_t* img, float (&x)[TOK]) { // tokens TOK g .. of channel v of a feature-major image
+#pragma unroll
+      for (int q = 0; q < TOK / 8; ++q)
+        unpack8(*reinterpret_cast<const uint4*>(img + sw128_offset(v, (TOK / 8) * g + q)),
+                *reinterpret_cast<float(*)[8]>(x + 8 * q));
+    };
+    float h[KC];                                         // h^T[v][KC g .. KC g + KC - 1]
     {
       const size_t base = ((size_t)n * p.HV + j) * 128 * 128 + v;
 #pragma unroll
-      for (int q = 0; q < 64; ++q) h[q] = p.h0 ? p.h0[base + (size_t)(64 * g + q) * 128] : 0.f;
+      for (int q = 0; q < KC; ++q) h[q] = p.h0 ? p.h0[base + (size_t)(KC * g + q) * 128] : 0.f;
     }
-    auto store_h = [&]() {                               // bf16 pairs of this thread's 64 key channels -> A operand
+    auto store_h = [&]() {                               // bf16 pairs of this thread's key channels -> A operand
 #pragma unroll
-      for (int c0 = 0; c0 < 64; c0 += 32) {
+      for (int c0 = 0; c0 < KC; c0 += 32) {
         uint32_t r[16];
 #pragma unroll
         for (int q = 0; q < 16; ++q) r[q] = pack_bf16(h[c0 + 2 * q], h[c0 + 2 * q + 1]);
-        tmem_st16(tmem + Cfg::TM_H + lane_base + 32 * g + c0 / 2, r);
+        tmem_st16(tmem + Cfg::TM_H + lane_base + (KC / 2) * g + c0 / 2, r);
       }
       tmem_st_wait();
     };
@@ -621,22 +641,18 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     auto output_part = [&](int c) {
       const int st = c % S;
       const uint8_t* stage = sm + st * Cfg::kStageB;
-      const int L = min(kChunk, len - c * kChunk);
-      float d[32];
-      ld32f(tmem + Cfg::TM_D1 + (c & 1) * 128 + lane_base + 64 + 32 * g, d);
-      float ol[32];
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        unpack8(*reinterpret_cast<const uint4*>(stage + Cfg::OFF_O + sw128_offset(v, 4 * g + q)),
-                *reinterpret_cast<float(*)[8]>(ol + 8 * q));
+      float d[TOK];
+      ld_cols(tmem + Cfg::TM_D1 + (c & 1) * 128 + lane_base + 64 + TOK * g, d);
+      float ol[TOK];
+      img_row(stage + Cfg::OFF_O, ol);
       mbar_arrive(&bar_empty[st]);                       // last read of the stage by this thread
-      // hand the 32 tokens of this thread's channel to the output warps (token-major tile, 2-byte stores: a warp
+      // hand the tokens of this thread's channel to the output warps (token-major tile, 2-byte stores: a warp
       // writes 64 contiguous bytes of a token row per instruction)
       uint8_t* tile = sm + Cfg::OFF_OUT + (c & 1) * 16384 + (v >> 6) * 8192 + (v & 7) * 2;
       named_sync(BAR_O_FREE + 2 * (c & 1), NCOMP + 64);  // the output warps are done with this tile's last contents
 #pragma unroll
-      for (int q = 0; q < 32; ++q) {
-        const int t = 32 * g + q;
+      for (int q = 0; q < TOK; ++q) {
+        const int t = TOK * g + q;
         *reinterpret_cast<__nv_bfloat16*>(tile + sw128_offset(t, (v & 63) >> 3)) =
             __float2bfloat16_rn(p.scale * (ol[q] + d[q]));
       }
@@ -651,25 +667,22 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
       HA_PROF(chain, 8 * c + 1);
       const float* sc = reinterpret_cast<const float*>(stage + Cfg::OFF_SC);
-      // U^T[v][32 g .. 32 g + 31], fetched while MMA1 runs
-      float u[32];
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        unpack8(*reinterpret_cast<const uint4*>(stage + Cfg::OFF_U + sw128_offset(v, 4 * g + q)),
-                *reinterpret_cast<float(*)[8]>(u + 8 * q));
+      float u[TOK];                                      // U^T[v][TOK g ..], fetched while MMA1 runs
+      img_row(stage + Cfg::OFF_U, u);
       mbar_wait(bar_mma1, ph, abort_flag);
       HA_PROF(chain, 8 * c + 2);
       tc_fence_after_sync();
       {
-        float d[32];
-        ld32f(tmem + Cfg::TM_D1 + (c & 1) * 128 + lane_base + 32 * g, d);
-        uint32_t r[16];
+        float d[TOK];
+        ld_cols(tmem + Cfg::TM_D1 + (c & 1) * 128 + lane_base + TOK * g, d);
+        uint32_t r[TOK / 2];
 #pragma unroll
-        for (int q = 0; q < 16; ++q) {
-          const float2 dc = *reinterpret_cast<const float2*>(sc + 32 * g + 2 * q);   // e^{G_L - G_i}, two tokens
+        for (int q = 0; q < TOK / 2; ++q) {
+          const float2 dc = *reinterpret_cast<const float2*>(sc + TOK * g + 2 * q);   // e^{G_L - G_i}, two tokens
           r[q] = pack_bf16((u[2 * q] - d[2 * q]) * dc.x, (u[2 * q + 1] - d[2 * q + 1]) * dc.y);
         }
-        tmem_st16(tmem + Cfg::TM_UT + lane_base + 16 * g, r);
+        if constexpr (TOK == 32) tmem_st16(tmem + Cfg::TM_UT + lane_base + 16 * g, r);
+        else tmem_st8(tmem + Cfg::TM_UT + lane_base + 8 * g, r);
         tmem_st_wait();
       }
       tc_fence_before_sync();
@@ -680,13 +693,13 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       HA_PROF(chain, 8 * c + 4);
       tc_fence_after_sync();
 #pragma unroll
-      for (int c0 = 0; c0 < 64; c0 += 32) {
+      for (int c0 = 0; c0 < KC; c0 += 32) {
         float d[32];
-        ld32f(tmem + Cfg::TM_D2 + lane_base + 64 * g + c0, d);
+        ld32f(tmem + Cfg::TM_D2 + lane_base + KC * g + c0, d);
         if constexpr (KDA) {
 #pragma unroll
           for (int q = 0; q < 32; q += 4) {
-            const float4 gm = *reinterpret_cast<const float4*>(sc + 64 + 64 * g + c0 + q);   // decay per key channel
+            const float4 gm = *reinterpret_cast<const float4*>(sc + 64 + KC * g + c0 + q);   // decay per key channel
             h[c0 + q] = fmaf(gm.x, h[c0 + q], d[q]);
             h[c0 + q + 1] = fmaf(gm.y, h[c0 + q + 1], d[q + 1]);
             h[c0 + q + 2] = fmaf(gm.z, h[c0 + q + 2], d[q + 2]);
@@ -709,7 +722,7 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     if (p.hT) {
       const size_t base = ((size_t)n * p.HV + j) * 128 * 128 + v;
 #pragma unroll
-      for (int q = 0; q < 64; ++q) p.hT[base + (size_t)(64 * g + q) * 128] = h[q];
+      for (int q = 0; q < KC; ++q) p.hT[base + (size_t)(KC * g + q) * 128] = h[q];
     }
   }
 
@@ -721,10 +734,10 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
   if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
 }
 
-template <bool KDA>
+template <bool KDA, int CG>
 cudaError_t run_t(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMap* mo, int grid, bool dependent,
                   cudaStream_t stream) {
-  auto kern = tc_chain_t_kernel<KDA>;
+  auto kern = tc_chain_t_kernel<KDA, CG>;
   constexpr int smem = ChainTCfg::kSmem;
   static_assert(smem <= 227 * 1024, "shared memory budget");
   if (!cp) {
@@ -735,7 +748,7 @@ cudaError_t run_t(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMa
   timer_mark(stream, "tc_chain");
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kTThreads);
+  cfg.blockDim = dim3(t_threads(CG));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -779,7 +792,9 @@ cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, const CUte
                         bool dependent, cudaStream_t stream) {
   if (nv == 32) return run_nv<32, KDA, 3, 1>(cp, mk, mo, grid, dependent, stream);
   if (nv == 64) return run_nv<64, KDA, 3, 2>(cp, mk, mo, grid, dependent, stream);
-  return run_t<KDA>(cp, mk, mo, grid, dependent, stream);      // all 128 channels: the whole-head kernel
+  // all 128 channels: the whole-head kernel (two column groups of compute warps; four measured no faster: its
+  // products, slowed by the shared-memory traffic around them, are the limit, not the epilogues)
+  return run_t<KDA, 2>(cp, mk, mo, grid, dependent, stream);
 }
 
 }  // namespace
