@@ -174,7 +174,7 @@ def test_tc_every_slice_width(nv, variant, monkeypatch):
     helpers.check_parity(inp)
 
 
-@pytest.mark.parametrize("case", ["gdn", "kda", "varlen", "gdn_nv64", "kda_nv64"])
+@pytest.mark.parametrize("case", ["gdn", "kda", "varlen", "gdn_nv64", "kda_nv64", "gdn_nv128", "kda_nv128"])
 def test_concurrent_prep_and_chain_mode(case, monkeypatch):
     """Concurrent mode (chosen by the launch planner while the chain CTAs need at most half of the SMs; forced
     here with HA_LA_TC_OVERLAP=2): the chain kernel runs next to the persistent prep kernel and takes each
@@ -188,6 +188,8 @@ def test_concurrent_prep_and_chain_mode(case, monkeypatch):
         w = synth.shrink(W["gdn_varlen"], seq_lens=[700, 0, 65, 1500], hk=2, hv=2)
     if case.endswith("nv64"):
         monkeypatch.setenv("HA_LA_TC_NV", "64")
+    if case.endswith("nv128"):                           # the whole-head kernel (state in tensor memory)
+        monkeypatch.setenv("HA_LA_TC_NV", "128")
     inp = synth.make_inputs(w, seed=37)
     monkeypatch.setenv("HA_LA_TC_OVERLAP", "0")
     o_seq, h_seq, st_seq = helpers.run_gpu(inp)
