@@ -478,14 +478,14 @@ def main():
     clocks["window"] = f"timed region, per-kernel timing and {time.perf_counter() - t_load:.2f} s of the same steps"
     kernel_ms = {k: float(np.mean(v)) for k, v in kt.items()}
     dom = max(kernel_ms, key=kernel_ms.get)
-    # algorithmic bytes each kernel is the one to touch ("Roofline accounting")
+    # algorithmic bytes each kernel is the one to touch: the prep kernel reads the inputs (q, k, v, g, beta),
+    # the chain kernel reads h0 and writes o and hT; the operand images between them are not algorithmic bytes
     e = 2 if w.dtype == "bf16" else 4
     in_bytes = T * (2 * w.hk * w.dk * e + w.hv * w.dv * e + w.hv * 4 * (1 + (w.dk if w.variant == "kda" else 1)))
     out_bytes = alg_bytes - in_bytes
     kernel_alg_bytes = {"simt_prefill": alg_bytes, "tc_prep": in_bytes, "tc_chain": out_bytes, "plan": 0.0}
-    # DRAM bytes per launch of that kernel from one ncu --set full capture of this workload
-    # (profiles/tc_prep_chain_gdn_layer_4k_ncu_full.md, profiles/tc_prep_chain_kda_8k_ncu_full.md,
-    # profiles/tc_prep_chain_nv64_gdn_gva_16k_ncu_full.md); cold-cache replays
+    # DRAM bytes per launch of that kernel from one ncu --set full capture of this workload (the summaries under
+    # profiles/ name the commands); cold-cache replays
     ncu_traffic = {("gdn_layer_4k", "tc_chain"): 84.71e6 + 5.90e6, ("gdn_layer_4k", "tc_prep"): 50.92e6 + 15.08e6,
                    ("kda_8k", "tc_prep"): 336.78e6 + 291.11e6, ("kda_8k", "tc_chain"): 338.73e6 + 56.62e6,
                    ("gdn_gva_16k", "tc_prep"): 272.71e6 + 487.64e6, ("gdn_gva_16k", "tc_chain"): 612.41e6 + 120.54e6}
