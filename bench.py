@@ -353,7 +353,7 @@ def decode_bench(args, rank, local_rank, world):
         dist.destroy_process_group()
 
 
-# DRAM bytes per launch of the decode kernel from its ncu capture (profiles/decode_gdn_decode_b256_ncu_full.md)
+# DRAM bytes per launch of the decode kernel from its ncu capture (summary under profiles/)
 DECODE_NCU_TRAFFIC = {"gdn_decode_b256": 271.69e6 + 211.84e6}
 
 
