@@ -339,3 +339,31 @@ def test_more_sequences_than_the_ranking_limit():
     pairs = [(n, 0) for n in sorted(set(range(0, 4500, 23)) | {1, 2, 4095, 4096, 4097, 4499, int(np.argmax(lens))})]
     res = helpers.check_parity(inp, pairs=pairs)
     print(res)
+
+
+def test_randomized_shapes_widths_and_modes(monkeypatch):
+    """Thirty seeded random cases: both variants, one to five sequences with lengths around the chunk
+    boundaries (empty ones included), grouped heads, three gate strengths, with and without an initial state,
+    every slice width of the chain kernel and every launch mode, against the oracle."""
+    import random
+
+    rng = random.Random(20260932114)
+    for it in range(30):
+        variant = rng.choice(["gdn", "kda"])
+        lens = [rng.choice([0, 1, 63, 64, 65, 127, 128, 129, 200, 511, 700, 1000, 1537, 2048])
+                for _ in range(rng.choice([1, 1, 2, 3, 5]))]
+        if sum(lens) == 0:
+            lens[0] = 77
+        hk = rng.choice([1, 2, 4])
+        hv = hk * rng.choice([1, 1, 2])
+        base = W["gdn_varlen"] if variant == "gdn" else W["kda_8k"]
+        w = synth.shrink(base, seq_lens=lens, hk=hk, hv=hv, gate_shift=rng.choice([-2.0, 0.0, 2.0]),
+                         h0_std=rng.choice([0.0, 0.02]), varlen=True)
+        inp = synth.make_inputs(w, seed=1000 + it)
+        for var, val in (("HA_LA_TC_NV", rng.choice(["", "32", "64", "128"])),
+                         ("HA_LA_TC_OVERLAP", rng.choice(["", "0", "2"]))):
+            if val:
+                monkeypatch.setenv(var, val)
+            else:
+                monkeypatch.delenv(var, raising=False)
+        helpers.check_parity(inp, scale=rng.choice([1.0, 0.5]))
