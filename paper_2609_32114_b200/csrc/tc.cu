@@ -105,7 +105,7 @@ int64_t next_epoch() {
 // needs an SM of its own, so the kernel's time is about  max(longest sequence, all sequences / SMs)  in chunk-times
 // when the lengths differ (more CTAs than SMs are started longest sequence first and pack well), and whole rounds
 // when they do not: with few chains the narrow slice wins, with many a wider one may.
-// Prep kernel: throughput-bound, about 3.45 (GDN) / 10.2 (KDA) SM-microseconds per (chunk, head), and never
+// Prep kernel: throughput-bound, about 3.45 (GDN) / 9.8 (KDA) SM-microseconds per (chunk, head), and never
 // faster than its rounds of one item per work group (3 per SM for GDN, 1 for KDA) at 9 / 10.5 us per item.
 // Back to back the two times add.  Concurrently (allowed while the chain's CTAs leave at least half of the SMs to
 // the prep kernel) the call takes the longer of the chain and of the prep kernel on the remaining SMs (plus some
@@ -123,7 +123,7 @@ TcPlan plan_tc(const Problem& p) {
   const double per_chunk_us[3] = {0.90, 1.23, 1.50};
   const bool kda = p.variant == HA_LA_KDA;
   auto prep_time = [&](int on_sms) {                     // the prep kernel on `on_sms` SMs
-    const double thru = items * (kda ? 10.2 : 3.45) / on_sms;
+    const double thru = items * (kda ? 9.8 : 3.45) / on_sms;
     const double groups = (double)on_sms * (kda ? 1 : 3);
     const double rounds = (double)(long long)((items + groups - 1) / groups) * (kda ? 10.5 : 9.0);
     return thru > rounds ? thru : rounds;

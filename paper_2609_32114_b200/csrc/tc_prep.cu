@@ -520,15 +520,14 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     tc_fence_before_sync();
     bsync();
     // ---- operands rescaled in place: K <- K 2^G (for W), Q <- Q 2^G (for Q~); K e^{G_L - G} for the chain.
-    // The tensor cores read the K+ / Q+ / K- copies, not these tiles, so this runs while they work -- unless a
-    // diagonal block has to be evaluated again from the raw tiles first.
-    auto rescale_pass = [&](bool all_warps) {            // by all 16 warps, or by the first 8 only
+    // The tensor cores read the K+ / Q+ / K- copies, not these tiles, so this runs while they work (on the helper
+    // warps) -- unless a diagonal block has to be evaluated again from the raw tiles first (then on the others).
+    auto rescale_pass = [&](int t) {                     // by eight warps; t = 0..255 within them
     {
-      const int i = all_warps ? tid >> 3 : tid >> 2;
-      const int nq = all_warps ? 2 : 4;
+      const int i = t >> 2;
 #pragma unroll 1
-      for (int q = 0; q < nq; ++q) {
-        const int cc = all_warps ? (tid & 7) + 8 * q : (tid & 3) + 4 * q;
+      for (int q = 0; q < 4; ++q) {
+        const int cc = (t & 3) + 4 * q;
         uint8_t* kt = sm + OFF_KQ + (cc >> 3) * 16384;
         const uint32_t off = sw128_offset(i, cc & 7);
         float kf[8], qf[8], gi[8], gl[8], kd[8];
@@ -571,13 +570,15 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     if (tid < 128) sQt[tid] = sGc[63 * LDG + tid];       // the chunk's total decay, for the chain kernel's scalars
     if (!anyfall) {
-      rescale_pass(true);
-      // That was the last use of the gate matrix (the scalars above are a copy), so the helper warps can fetch
-      // the next item's gate rows into it right away, while the other warps solve: a warp needs some 3 k cycles
-      // to issue its 64 row copies, which the whole group used to wait for at the top of the next item.
+      // The helper warps rescale the tiles on their own while the other warps take the first product's result and
+      // solve (nothing there reads the tiles; the W / U products, much later, wait at barrier 10).  That is the
+      // last use of the gate matrix (the scalars above are a copy), so the helpers then fetch the next item's gate
+      // rows into it right away: a warp needs some 3 k cycles to issue its 64 row copies, which the whole group
+      // used to wait for at the top of the next item.
       if (is_main) {
         asm volatile("bar.arrive 9, %0;" ::"r"(kKdaThreads) : "memory");
       } else {
+        rescale_pass(tid - kPrepThreads);
         // the helpers' part of the rescaled K / Q / K e^{G_L-G} tiles: visible to the tensor cores and the bulk
         // stores (proxy fence) once the other warps have passed barrier 10, before the W / U products
         fence_proxy_async_smem();
@@ -663,7 +664,7 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       gsync();                                   // everyone is done with the raw K and Q tiles
-      rescale_pass(false);
+      rescale_pass(tid);
     }
     }  // is_main
 
