@@ -749,25 +749,55 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   PP(5);
 
   // ---- op #3 Solve: T = (I + A)^-1
-  if (tid < 64) {
-    // Four 16x16 diagonal blocks; thread = (block, column c of the inverse), fp32 forward substitution row by
-    // row: y_q = [q == c] - sum_{r<q} A[q][r] y_r.  The inverse goes to a scratch copy first (the other
-    // threads of the block are still reading A).
-    const int blk = tid >> 4, c = tid & 15, o = blk * 16;
-    float y[16];
+  {
+    // Four 16x16 diagonal blocks, each as 2 x 2 blocks of 8 x 8:  [[X11, 0], [X21, X22]]  with
+    // X11 = (I + A11)^-1, X22 = (I + A22)^-1 by fp32 forward substitution (64 threads: block, half, column; eight
+    // steps instead of sixteen), then X21 = -X22 (A21 X11) by all threads, one element each.  The inverse goes to
+    // a scratch copy first (other threads are still reading A).
+    float* sM = reinterpret_cast<float*>(sD + 4 * 256);   // fp32 [4][8][8]: A21 X11
+    if (tid < 64) {
+      const int blk = tid >> 4, hb = (tid >> 3) & 1, c = tid & 7, o = blk * 16 + hb * 8;
+      __half* dst = sD + blk * 256 + (hb * 8) * 16 + hb * 8 + c;
+      float y[8];
 #pragma unroll
-    for (int q = 0; q < 16; ++q) {
-      float a[16];
-      if (q > 0) unpack8h(*reinterpret_cast<const uint4*>(sAh + (o + q) * LDH + o), *reinterpret_cast<float(*)[8]>(a));
-      if (q > 8) unpack8h(*reinterpret_cast<const uint4*>(sAh + (o + q) * LDH + o + 8), *reinterpret_cast<float(*)[8]>(a + 8));
-      float s0 = q == c ? 1.f : 0.f, s1 = 0.f;
+      for (int q = 0; q < 8; ++q) {
+        float a[8];
+        if (q > 0) unpack8h(*reinterpret_cast<const uint4*>(sAh + (o + q) * LDH + o), a);
+        float s0 = q == c ? 1.f : 0.f, s1 = 0.f;
 #pragma unroll
-      for (int r = 0; r < q; ++r) {
-        if (r & 1) s1 = fmaf(-a[r], y[r], s1);
-        else s0 = fmaf(-a[r], y[r], s0);
+        for (int r = 0; r < q; ++r) {
+          if (r & 1) s1 = fmaf(-a[r], y[r], s1);
+          else s0 = fmaf(-a[r], y[r], s0);
+        }
+        y[q] = s0 + s1;
+        dst[q * 16] = __float2half_rn(y[q]);
+        if (hb == 0) sD[blk * 256 + q * 16 + 8 + c] = __float2half_rn(0.f);   // the block above the diagonal
       }
-      y[q] = s0 + s1;
-      sD[blk * 256 + q * 16 + c] = __float2half_rn(y[q]);
+    }
+    gsync();
+    const int blk = tid >> 6, bi = (tid >> 3) & 7, bj = tid & 7, o = blk * 16;
+    {
+      float a[8];
+      unpack8h(*reinterpret_cast<const uint4*>(sAh + (o + 8 + bi) * LDH + o), a);        // row bi of A21
+      float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; k += 2) {
+        m0 = fmaf(a[k], __half2float(sD[blk * 256 + k * 16 + bj]), m0);                   // column bj of X11
+        m1 = fmaf(a[k + 1], __half2float(sD[blk * 256 + (k + 1) * 16 + bj]), m1);
+      }
+      sM[tid] = m0 + m1;
+    }
+    gsync();
+    {
+      float x[8];
+      unpack8h(*reinterpret_cast<const uint4*>(sD + blk * 256 + (8 + bi) * 16 + 8), x);   // row bi of X22
+      float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; k += 2) {
+        m0 = fmaf(x[k], sM[blk * 64 + k * 8 + bj], m0);
+        m1 = fmaf(x[k + 1], sM[blk * 64 + (k + 1) * 8 + bj], m1);
+      }
+      sD[blk * 256 + (8 + bi) * 16 + bj] = __float2half_rn(-(m0 + m1));
     }
   }
   gsync();
