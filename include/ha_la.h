@@ -41,7 +41,25 @@
  *     not matter and nothing in it needs clearing, but calls that may overlap on
  *     the GPU (different streams without an ordering) need a workspace each.
  *   - Sequence lengths need not be multiples of 64; length-0 sequences are
- *     legal (hT = h0).  Log-gates are expected to be <= 0.
+ *     legal (hT = h0).
+ *
+ * What the inputs must satisfy
+ *   - Every value is finite.  Log-gates are <= 0 (the kernels evaluate decays only
+ *     as exp of non-positive numbers; a positive log-gate gives unspecified results).
+ *   - d_k == d_v (64 or 128).
+ *   - The tensor-core path (bf16, d = 128) holds (I + A)^-1 of operator #3 in fp16
+ *     between the levels of its blocked solve.  That is exact enough whenever
+ *     beta |k|^2 stays within the delta rule's own stability range (<= 2; keys of
+ *     norm 0.5 .. 2 are tested).  Inputs far outside it can overflow the fp16 range;
+ *     the kernel detects that and reports HA_LA_ERR_DEVICE_CHECK through status_word
+ *     instead of returning wrong numbers silently.
+ *
+ * Environment switches (test hooks, read by the host launch code; they change how the
+ * work is launched, never the result): HA_LA_FORCE_SIMT=1 (read once) sends every shape
+ * to the fp32 CUDA-core kernel; HA_LA_TC_NV=32|64|128 fixes the slice width of the
+ * sequential kernel; HA_LA_TC_OVERLAP=0|2 forbids / forces running the two tensor-core
+ * kernels side by side; HA_LA_TC_SEGMENTS=1|2|4 fixes the number of segments a head's
+ * chunk sequence is split into.  Production callers leave them unset.
  */
 #ifndef HA_LA_H_
 #define HA_LA_H_
@@ -137,7 +155,7 @@ int ha_la_prefill_timed(const ha_la_prefill_args* args, void* cuda_stream, int m
  * counterpart of this entry point; it computes exactly what ha_la_prefill computes.
  *
  *   - args->workspace and args->workspace_bytes are ignored.  The chunk table lives in a fixed
- *     array inside the library image (ha_la_prefill_noalloc_scratch_bytes() bytes, about 212 KiB),
+ *     array inside the library image (ha_la_prefill_noalloc_scratch_bytes() bytes, 209 KiB),
  *     which every GPU that loads the library holds until the process exits.
  *   - Limits: at most 1024 sequences (batch rows or packed sequences) and at most 16384 chunk
  *     slots ((seqlen + 63 * num_seqs) / 64 in packed mode, batch * ceil(seqlen / 64) otherwise);
@@ -147,7 +165,9 @@ int ha_la_prefill_timed(const ha_la_prefill_args* args, void* cuda_stream, int m
  *     library's tolerances.
  *   - It calls no cudaMalloc / cudaFree and no allocating library routine.  Its FIRST call on a
  *     device looks up the array's device address (cudaGetSymbolAddress, with that device current)
- *     and caches it; make that first call outside any stream capture.
+ *     and caches it; make that first call outside any stream capture.  The cached address belongs
+ *     to the device's primary context: it does not survive cudaDeviceReset, and a context other
+ *     than the primary one on the same device ordinal must not use this entry point.
  *   - All calls on a device share the one array.  Nothing in it has to start at zero (each call
  *     rewrites every entry it later reads), but two calls that overlap on the GPU -- different
  *     streams without an ordering between them -- race on it: serialise them.                     */
@@ -155,9 +175,9 @@ int ha_la_prefill_noalloc(const ha_la_prefill_args* args, void* cuda_stream);
 size_t ha_la_prefill_noalloc_scratch_bytes(void);
 
 /* One decoding step of the same layer: ONE new token per sequence, the recurrent state kept by the
- * caller between calls.  The paper hands "updated states for downstream layers and subsequent
- * decoding" from the prefill to the decoder (Section "HA-NPU overview") and leaves the decoding
- * step itself to the framework's native backend; this entry point is that step for the state
+ * caller between calls.  In the paper the prefill's online stage returns the updated state so that
+ * later layers and the decoder can carry on from it (Section "HA-NPU overview"), and the decoding
+ * step itself is left to the framework's native backend; this entry point is that step for the state
  * layout ha_la_prefill produces (hT), so that prefill and decode share one library.
  *
  * For every sequence n and V-head j (QK-head jq = j / (HV/HK)), with h = h_in[n,j] (zeros if NULL):

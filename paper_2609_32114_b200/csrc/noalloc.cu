@@ -12,29 +12,36 @@
 // cudaGetSymbolAddress, with that device current, on the entry point's first call on that device.
 #include "common.cuh"
 
+#include <atomic>
+
 namespace ha_la {
 namespace {
 
 constexpr int kMaxSeqs = 1024;        // sequences (batch rows or packed sequences)
 constexpr int kMaxChunks = 16384;     // chunk slots: about one million tokens
 constexpr size_t kScratchInts = 8 + 3 * (size_t)kMaxSeqs + (kMaxSeqs + 1) + 3 * (size_t)kMaxChunks;
-constexpr size_t kScratchBytes = (kScratchInts * sizeof(int32_t) + 255) / 256 * 256;   // 212 KiB
+// rounded like plan_bytes() (to 1 KiB), so that a problem at exactly both limits fits: 209 KiB
+constexpr size_t kScratchBytes = (kScratchInts * sizeof(int32_t) + 1023) / 1024 * 1024;
 
 static __device__ __align__(256) unsigned char g_plan_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {};   // device address of g_plan_scratch on each device, once known
+// Device address of g_plan_scratch on each device, once known.  Host threads may race on a slot: every writer
+// stores the same value (the address is a property of the device's primary context), so the race is between
+// equal stores; the slots are atomics only to make that well defined.  A cached address belongs to the
+// device's primary context and does not survive cudaDeviceReset.
+std::atomic<void*> g_scratch_addr[kMaxDevices];
 
 // Looks the array's device address up (first call on this device) or returns the cached one.
 int scratch_address(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HA_LA_ERR_CUDA;
-  if (!g_scratch_addr[dev]) {
-    void* p = nullptr;
+  void* p = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!p) {
     if (cudaGetSymbolAddress(&p, g_plan_scratch) != cudaSuccess || !p) return HA_LA_ERR_CUDA;
-    g_scratch_addr[dev] = p;
+    g_scratch_addr[dev].store(p, std::memory_order_release);
   }
-  *out = g_scratch_addr[dev];
+  *out = p;
   return HA_LA_OK;
 }
 
@@ -49,14 +56,7 @@ extern "C" int ha_la_prefill_noalloc(const ha_la_prefill_args* a, void* cuda_str
   size_t unused = 0;
   const int rc = ha_la_prefill_workspace_bytes(a, &unused);
   if (rc != HA_LA_OK) return rc;
-  if (!a->q || !a->k || !a->v || !a->g || !a->beta || !a->o) return HA_LA_ERR_INVALID_ARG;
   const bool packed = a->num_seqs > 0 || a->cu_seqlens;
-  if (packed && !a->cu_seqlens) return HA_LA_ERR_INVALID_ARG;
-  const uintptr_t al16 = (uintptr_t)a->q | (uintptr_t)a->k | (uintptr_t)a->v | (uintptr_t)a->o |
-                         (uintptr_t)a->h0 | (uintptr_t)a->hT;
-  if (al16 & 15) return HA_LA_ERR_INVALID_ARG;
-  if (((uintptr_t)a->g | (uintptr_t)a->beta | (uintptr_t)a->cu_seqlens | (uintptr_t)a->status_word) & 3)
-    return HA_LA_ERR_INVALID_ARG;
 
   Problem p;
   p.variant = a->variant; p.dtype = a->dtype;
@@ -74,7 +74,15 @@ extern "C" int ha_la_prefill_noalloc(const ha_la_prefill_args* a, void* cuda_str
   }
   p.max_seq_chunks = (p.max_len + kChunk - 1) / kChunk;
   if (!simt_supported(p)) return HA_LA_ERR_UNSUPPORTED;
+  // sizes first (shapes alone decide them), then the pointers
   if (p.N > kMaxSeqs || p.max_chunks > kMaxChunks || plan_bytes(p) > kScratchBytes) return HA_LA_ERR_TOO_LARGE;
+  if (!a->q || !a->k || !a->v || !a->g || !a->beta || !a->o) return HA_LA_ERR_INVALID_ARG;
+  if (packed && !a->cu_seqlens) return HA_LA_ERR_INVALID_ARG;
+  const uintptr_t al16 = (uintptr_t)a->q | (uintptr_t)a->k | (uintptr_t)a->v | (uintptr_t)a->o |
+                         (uintptr_t)a->h0 | (uintptr_t)a->hT;
+  if (al16 & 15) return HA_LA_ERR_INVALID_ARG;
+  if (((uintptr_t)a->g | (uintptr_t)a->beta | (uintptr_t)a->cu_seqlens | (uintptr_t)a->status_word) & 3)
+    return HA_LA_ERR_INVALID_ARG;
 
   void* scratch = nullptr;
   const int src = scratch_address(&scratch);

@@ -835,6 +835,16 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int i = tid >> 2, q4 = tid & 3;                // row, quarter (16 columns = two 16-byte pieces)
     const uint4 traw0 = *reinterpret_cast<const uint4*>(sAh + i * LDH + q4 * 16);
     const uint4 traw1 = *reinterpret_cast<const uint4*>(sAh + i * LDH + q4 * 16 + 8);
+    {
+      // T left the fp16 range (an exponent field of all ones: infinity or NaN) only for inputs far outside the
+      // delta rule's stable range (beta |k|^2 <= 2): report it instead of returning wrong numbers silently.
+      const uint32_t w[8] = {traw0.x, traw0.y, traw0.z, traw0.w, traw1.x, traw1.y, traw1.z, traw1.w};
+      bool bad = false;
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        bad |= (w[e] & 0x7c000000u) == 0x7c000000u || (w[e] & 0x00007c00u) == 0x00007c00u;
+      if (bad) report_status(p.status, HA_LA_ERR_DEVICE_CHECK);
+    }
     gsync();
 #pragma unroll
     for (int q = 0; q < 2; ++q) {

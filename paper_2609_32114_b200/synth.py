@@ -51,7 +51,7 @@ class Workload:
     index: int = 0               # stream selector
 
 
-# The five workloads of the north-star specification.
+# The five benchmark workloads.
 WORKLOADS = {
     "gdn_fp32_small": Workload("gdn_fp32_small", "gdn", "fp32", 1, 1, 64, 64, seq_lens=(256,), index=0),
     "gdn_layer_4k": Workload("gdn_layer_4k", "gdn", "bf16", 16, 16, 128, 128, seq_lens=(4096,),

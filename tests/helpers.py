@@ -1,8 +1,8 @@
 """Shared helpers of the GPU parity tests: run the CUDA library and the CPU oracle on the same
-seeded inputs and compare with the spec error metric."""
+seeded inputs and compare with the stated error metric (max-norm relative error per output tensor)."""
 import numpy as np
 
-TOL = {"bf16": 2e-2, "fp32": 1e-4}     # max|err| / max|ref|, per output tensor (spec tolerances)
+TOL = {"bf16": 2e-2, "fp32": 1e-4}     # max|err| / max|ref|, per output tensor (the stated tolerances)
 
 
 def to_device(inp, device="cuda"):

@@ -40,6 +40,11 @@ def _both(inp):
     assert np.isfinite(o_a).all() and np.isfinite(h_a).all()
     assert np.abs(o_a - o_b).max() <= tol * np.abs(o_b).max()
     assert np.abs(h_a - h_b).max() <= tol * np.abs(h_b).max()
+    # ... and against the CPU oracle (with bf16 inputs and d = 128 ha_la_prefill runs the tensor-core kernels,
+    # so this entry point is the only caller of the CUDA-core kernel for that shape)
+    o_orc, h_orc = helpers.run_oracle(inp)
+    assert helpers.rel_max_err(o_a.reshape(o_orc.shape), o_orc) <= tol
+    assert helpers.rel_max_err(h_a.reshape(h_orc.shape), h_orc) <= tol
 
 
 def test_noalloc_matches_prefill_twice_in_a_row():
@@ -66,4 +71,18 @@ def test_noalloc_rejects_problems_beyond_its_scratch():
     assert "scratch" in ha.status_string(binding.HA_LA_ERR_TOO_LARGE)
     a = ha.make_args(variant="gdn", dtype="bf16", batch=1, seqlen=4096, hk=1, hv=1, dk=64, dv=64, num_seqs=2000,
                      q=4096, k=4096, v=4096, g=4096, beta=4096, o=8192, cu_seqlens=4096)
+    assert ha.ha_la_prefill_noalloc(a) == binding.HA_LA_ERR_TOO_LARGE
+
+
+def test_noalloc_accepts_its_documented_limits():
+    """Exactly 1024 sequences and 16384 chunk slots is inside the documented limits: the size check must pass
+    (the call is then refused for its null pointers, before anything is launched)."""
+    import paper_2609_32114_b200 as ha
+    from paper_2609_32114_b200 import binding
+
+    seqlen = 16384 * 64 - 63 * 1024                    # (seqlen + 63 * num_seqs) / 64 == 16384 chunk slots
+    a = ha.make_args(variant="gdn", dtype="bf16", batch=1, seqlen=seqlen, hk=1, hv=1, dk=64, dv=64, num_seqs=1024)
+    assert ha.ha_la_prefill_noalloc(a) == binding.HA_LA_ERR_INVALID_ARG      # null q, k, ...: sizes were accepted
+    a = ha.make_args(variant="gdn", dtype="bf16", batch=1, seqlen=seqlen + 64, hk=1, hv=1, dk=64, dv=64,
+                     num_seqs=1024, q=4096, k=4096, v=4096, g=4096, beta=4096, o=8192, cu_seqlens=4096)
     assert ha.ha_la_prefill_noalloc(a) == binding.HA_LA_ERR_TOO_LARGE
