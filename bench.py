@@ -12,8 +12,11 @@ over one batch of the synthetic workload.  Prints ONE JSON line (rank 0).
 * e2e          : the same metric through the public API with HOST buffers: pinned host -> device
                  copies of every input and device -> host copies of o and hT inside the timed region.
 * roofline     : for the dominant kernel, timed live with CUDA events between kernels
-                 (ha_la_prefill_timed); `path` gives the spec whole-path figure
-                 (slower of FLOPs at the measured bf16 peak and bytes at the measured HBM rate).
+                 (ha_la_prefill_timed): the path's algorithmic bytes over that kernel's time over the
+                 measured HBM rate; `path` gives the whole-call figure (slower of FLOPs at the measured
+                 bf16 peak and bytes at the measured HBM rate, over the time of the whole call).
+* parity       : o and hT of the last timed step against the fp64 oracle (all heads), same run; a result
+                 outside the stated tolerance makes the run fail.
 * cpu_baseline : the fp64 oracle, as it stands, on this machine's host cores, on a bounded sample.
 * --impl reference : times only the oracle (rank 0) and prints its line with "impl": "reference".
 
@@ -39,6 +42,21 @@ from paper_2609_32114_b200 import synth  # noqa: E402
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 METRIC = "LA-layer prefill tokens/s"
+
+
+def load_traffic():
+    """DRAM bytes per launch of each profiled kernel (profiles/traffic.json, written from the ncu summaries by
+    `python -m paper_2609_32114_b200.ncu_summary traffic`)."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(p):
+        return {}
+    with open(p) as f:
+        return json.load(f)
+
+
+def ncu_traffic(workload: str, kernel: str):
+    e = load_traffic().get(workload, {}).get(kernel)
+    return None if e is None else e["dram_read"] + e["dram_write"]
 
 
 def load_peaks():
@@ -329,7 +347,7 @@ def decode_bench(args, rank, local_rank, world):
         achieved = alg_bytes / sec / 1e9
         roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                    "traffic": DECODE_NCU_TRAFFIC.get(args.workload), "kernel_alg_bytes": alg_bytes,
+                    "traffic": ncu_traffic(args.workload, "decode"), "kernel_alg_bytes": alg_bytes,
                     "peak_source": peaks["source"], "kernel_ms": {"decode_kernel": ms_per_step},
                     "path": {"bound": "hbm", "roofline_us": 1e6 * alg_bytes / (peaks["hbm_gbs"] * 1e9),
                              "measured_us": 1e3 * ms_per_step, "frac": achieved / peaks["hbm_gbs"],
@@ -353,18 +371,158 @@ def decode_bench(args, rank, local_rank, world):
         dist.destroy_process_group()
 
 
-# DRAM bytes per launch of the decode kernel from its ncu capture (summary under profiles/)
-DECODE_NCU_TRAFFIC = {"gdn_decode_b256": 271.69e6 + 211.84e6}
+def measure(ha, helpers, w, inp, steps, warmup, dev, local_rank, dist, peaks, world, sample_clocks=True):
+    """Device-timed steps of ha_la_prefill on workload `w`: `steps` timed calls after max(warmup, 3) untimed ones,
+    one CUDA-event pair per step on the launching stream, every step on a different resident input/output set."""
+    import torch
+
+    T, N = inp["T"], inp["N"]
+    alg_bytes = synth.algorithmic_bytes(w, T, N)
+    alg_flops = synth.algorithmic_flops(w, T)
+    # R resident buffer sets, total > 2 x L2, visited round-robin
+    base = helpers.to_device(inp, dev)
+    R = max(2, int(np.ceil(2.2 * L2_BYTES / alg_bytes)) + 1)
+    R = min(R, 8)
+    sets = []
+    shared_ws = None                                     # the workspace is the caller's scratch: one for all sets
+    for r in range(R):
+        d = base if r == 0 else {k: (v.clone() if hasattr(v, "clone") else v) for k, v in base.items()}
+        a, keep = ha.prepare_args(d["q"], d["k"], d["v"], d["g"], d["beta"], variant=w.variant, h0=d["h0"],
+                                  cu_seqlens=d["cu_seqlens"], max_seqlen=d["max_seqlen"], workspace=shared_ws)
+        shared_ws = keep["workspace"]
+        sets.append((a, keep))
+    flush = None
+    if R * alg_bytes < 2 * L2_BYTES:
+        flush = torch.empty(3 * L2_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    sptr = stream.cuda_stream
+
+    def step(i):
+        rc = ha.ha_la_prefill_raw(sets[i % R][0], sptr)
+        if rc != 0:
+            raise ha.HaLaError(rc, "ha_la_prefill")
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def check_status(when):
+        for a, keep in sets:
+            st = int(keep["status_word"].item())
+            if st != 0:
+                raise SystemExit(f"device status word = {st} ({ha.status_string(st)}) {when}")
+
+    for i in range(max(warmup, 3)):
+        step(i)
+    barrier()
+    check_status("during warm-up")
+
+    # ---- timed region: exactly `steps` steps, device-timed per step (flush, if any, sits outside the events)
+    sampler = ClockSampler(local_rank) if sample_clocks else None
+    if sampler:
+        sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    barrier()
+    t_wall = time.perf_counter()
+    for i in range(steps):
+        if flush is not None:
+            flush.fill_(i & 0xff)
+        evs[i][0].record(stream)
+        step(i)
+        evs[i][1].record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    check_status("during the timed steps")
+    last = sets[(steps - 1) % R][1]
+    last_out = {"o": last["o"].clone(), "hT": last["hT"].clone()}     # what the last timed step wrote
+    step_ms = [a.elapsed_time(b) for a, b in evs]
+    total_ms = max_over_ranks(dist, float(np.sum(step_ms)), dev)
+    ms_per_step = total_ms / steps
+    value = job_throughput(world, T, ms_per_step)
+
+    # ---- per-kernel device time (events between kernels), averaged over a few cold-L2 steps
+    kt = {}
+    for i in range(min(steps, 8)):
+        if flush is not None:
+            flush.fill_(i)
+        for name, ms in ha.ha_la_prefill_timed(sets[(i + 1) % R][0], sptr):
+            kt.setdefault(name, []).append(ms)
+    clocks = None
+    if sampler:
+        # nvidia-smi samples every ~100 ms: if the timed region was shorter than a few samples, keep the same
+        # steps running (untimed) until some have been taken under this load
+        t_load = time.perf_counter()
+        i = 0
+        while len(sampler.rows) < 4 and time.perf_counter() - t_load < 2.0:
+            for _ in range(16):
+                step(i)
+                i += 1
+            barrier()
+        clocks = sampler.stop()
+        clocks["window"] = (f"timed region ({t_wall * 1e3:.0f} ms), per-kernel timing and "
+                            f"{time.perf_counter() - t_load:.2f} s of the same steps")
+    kernel_ms = {k: float(np.mean(v)) for k, v in kt.items()}
+    dom = max(kernel_ms, key=kernel_ms.get)
+    # per-kernel attribution: the algorithmic bytes each kernel is the one to touch (the prep kernel reads q, k, v,
+    # g, beta; the chain kernel reads h0 and writes o and hT; the operand images between them are not algorithmic)
+    e = 2 if w.dtype == "bf16" else 4
+    in_bytes = T * (2 * w.hk * w.dk * e + w.hv * w.dv * e + w.hv * 4 * (1 + (w.dk if w.variant == "kda" else 1)))
+    kernel_alg_bytes = {"simt_prefill": alg_bytes, "tc_prep": in_bytes, "tc_chain": alg_bytes - in_bytes, "plan": 0.0}
+    dom_s = kernel_ms[dom] / 1e3
+    achieved = alg_bytes / dom_s / 1e9                   # the path's bytes over the dominant kernel's time
+    t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_flop = alg_flops / (peaks["bf16_tflops"] * 1e12)
+    path_s = ms_per_step / 1e3
+    nv_plan, conc_plan = ha.ha_la_prefill_launch_plan(sets[0][0])
+    launch_mode = ("fp32 CUDA-core kernel" if nv_plan == 0 else
+                   f"{nv_plan}-channel slices, prep and chain kernels " + ("side by side" if conc_plan else "back to back"))
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic(w.name, dom),
+                "alg_bytes": alg_bytes, "peak_source": peaks["source"],
+                "kernel_ms": kernel_ms,      # each kernel alone (sequential launches with events in between)
+                "per_kernel": {k: {"alg_bytes_it_touches": kernel_alg_bytes.get(k, 0.0),
+                                   "achieved_gbs": kernel_alg_bytes.get(k, 0.0) / (v / 1e3) / 1e9 if v > 0 else None,
+                                   "traffic": ncu_traffic(w.name, k)} for k, v in kernel_ms.items()},
+                # what the timed steps used (kernel_ms is always back to back, and then with the planner's
+                # back-to-back slice width, which may differ)
+                "launch_mode": launch_mode,
+                "path": {"bound": "hbm" if t_hbm >= t_flop else "tensor", "roofline_us": 1e6 * max(t_hbm, t_flop),
+                         "measured_us": 1e6 * path_s, "frac": max(t_hbm, t_flop) / path_s,
+                         "achieved_gbs": alg_bytes / path_s / 1e9, "achieved_tflops": alg_flops / path_s / 1e12,
+                         "alg_bytes": alg_bytes, "alg_flops": alg_flops}}
+    return dict(sets=sets, R=R, base=base, stream=stream, sptr=sptr, ms_per_step=ms_per_step, value=value,
+                ms_median=float(np.median(step_ms)), ms_min=float(np.min(step_ms)), ms_max=float(np.max(step_ms)),
+                roofline=roofline, clocks=clocks, alg_bytes=alg_bytes, wall_s=t_wall, check_status=check_status,
+                last_out=last_out, flushed=flush is not None,
+                launches_per_step=ha.ha_la_prefill_num_launches(sets[0][0]), path=ha.ha_la_prefill_path(sets[0][0]))
+
+
+def parity_of(helpers, inp, out):
+    """o and hT in `out` (device tensors a step wrote) against the oracle on every (sequence, V-head) pair."""
+    w = inp["workload"]
+    o = out["o"].float().cpu().numpy().reshape(inp["T"], w.hv, w.dv)
+    hT = out["hT"].cpu().numpy().astype(np.float64)
+    o_ref, hT_ref = helpers.run_oracle(inp)
+    tol = helpers.TOL[w.dtype]
+    res = {"o_err": helpers.rel_max_err(o, o_ref), "hT_err": helpers.rel_max_err(hT, hT_ref),
+           "o_nmse": helpers.nmse(o, o_ref), "hT_nmse": helpers.nmse(hT, hT_ref), "tolerance": tol,
+           "metric": "max|err| / max|ref| per tensor, all heads, outputs of the last timed step"}
+    res["ok"] = bool(np.isfinite(o).all() and np.isfinite(hT).all() and res["o_err"] <= tol and res["hT_err"] <= tol)
+    return res
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="gdn_layer_4k", choices=sorted(synth.WORKLOADS) + sorted(DECODE_WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-parity", action="store_true", help="skip the oracle comparison of the timed outputs")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the short timings of the other workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -397,34 +555,11 @@ def main():
     # every rank draws its own batch of the same workload (weak scaling over independent batches)
     inp = synth.make_inputs(w, seed=rank_seed(rank))
     T, N = inp["T"], inp["N"]
-    alg_bytes = synth.algorithmic_bytes(w, T, N)
-    alg_flops = synth.algorithmic_flops(w, T)
     peaks = load_peaks()
-
-    # R resident buffer sets, total > 2 x L2, visited round-robin
-    base = helpers.to_device(inp, dev)
-    R = max(2, int(np.ceil(2.2 * L2_BYTES / alg_bytes)) + 1)
-    R = min(R, 8)
-    sets = []
-    shared_ws = None                                     # the workspace is the caller's scratch: one for all sets
-    for r in range(R):
-        d = base if r == 0 else {k: (v.clone() if hasattr(v, "clone") else v) for k, v in base.items()}
-        a, keep = ha.prepare_args(d["q"], d["k"], d["v"], d["g"], d["beta"], variant=w.variant, h0=d["h0"],
-                                  cu_seqlens=d["cu_seqlens"], max_seqlen=d["max_seqlen"], workspace=shared_ws)
-        shared_ws = keep["workspace"]
-        sets.append((a, keep))
-    flush = None
-    if R * alg_bytes < 2 * L2_BYTES:
-        flush = torch.empty(3 * L2_BYTES, dtype=torch.uint8, device=dev)
-    stream = torch.cuda.current_stream(dev)
-    sptr = stream.cuda_stream
-    launches_per_step = ha.ha_la_prefill_num_launches(sets[0][0])
-    path = ha.ha_la_prefill_path(sets[0][0])
-
-    def step(i):
-        rc = ha.ha_la_prefill_raw(sets[i % R][0], sptr)
-        if rc != 0:
-            raise ha.HaLaError(rc, "ha_la_prefill")
+    m = measure(ha, helpers, w, inp, args.steps, args.warmup, dev, local_rank, dist, peaks, world)
+    sets, R, base, stream, sptr = m["sets"], m["R"], m["base"], m["stream"], m["sptr"]
+    ms_per_step, value, roofline, clocks = m["ms_per_step"], m["value"], m["roofline"], m["clocks"]
+    alg_bytes = m["alg_bytes"]
 
     def barrier():
         torch.cuda.synchronize(dev)
@@ -432,83 +567,10 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    for i in range(max(args.warmup, 3)):
-        step(i)
-    barrier()
-    for a, keep in sets:
-        assert int(keep["status_word"].item()) == 0, "device status word set during warm-up"
-
-    # ---- timed region: exactly K steps, device-timed per step (flush, if any, sits outside the events)
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    barrier()
-    t_wall = time.perf_counter()
-    for i in range(args.steps):
-        if flush is not None:
-            flush.fill_(i & 0xff)
-        evs[i][0].record(stream)
-        step(i)
-        evs[i][1].record(stream)
-    barrier()
-    t_wall = time.perf_counter() - t_wall
-    step_ms = [a.elapsed_time(b) for a, b in evs]
-    total_ms = max_over_ranks(dist, float(np.sum(step_ms)), dev)
-    ms_per_step = total_ms / args.steps
-    value = job_throughput(world, T, ms_per_step)
-
-    # ---- per-kernel device time (events between kernels), averaged over a few cold-L2 steps
-    kt = {}
-    reps = min(args.steps, 8)
-    for i in range(reps):
-        if flush is not None:
-            flush.fill_(i)
-        for name, ms in ha.ha_la_prefill_timed(sets[(i + 1) % R][0], sptr):
-            kt.setdefault(name, []).append(ms)
-    # nvidia-smi cannot sample faster than every ~100 ms and a timed region of K short steps is over before
-    # its first sample: keep the same steps running (untimed) until a few samples have been taken under this load.
-    t_load = time.perf_counter()
-    i = 0
-    while len(sampler.rows) < 4 and time.perf_counter() - t_load < 2.0:
-        for _ in range(16):
-            step(i)
-            i += 1
-        barrier()
-    clocks = sampler.stop()
-    clocks["window"] = f"timed region, per-kernel timing and {time.perf_counter() - t_load:.2f} s of the same steps"
-    kernel_ms = {k: float(np.mean(v)) for k, v in kt.items()}
-    dom = max(kernel_ms, key=kernel_ms.get)
-    # algorithmic bytes each kernel is the one to touch: the prep kernel reads the inputs (q, k, v, g, beta),
-    # the chain kernel reads h0 and writes o and hT; the operand images between them are not algorithmic bytes
-    e = 2 if w.dtype == "bf16" else 4
-    in_bytes = T * (2 * w.hk * w.dk * e + w.hv * w.dv * e + w.hv * 4 * (1 + (w.dk if w.variant == "kda" else 1)))
-    out_bytes = alg_bytes - in_bytes
-    kernel_alg_bytes = {"simt_prefill": alg_bytes, "tc_prep": in_bytes, "tc_chain": out_bytes, "plan": 0.0}
-    # DRAM bytes per launch of that kernel from one ncu --set full capture of this workload (the summaries under
-    # profiles/ name the commands); cold-cache replays
-    ncu_traffic = {("gdn_layer_4k", "tc_chain"): 84.71e6 + 5.90e6, ("gdn_layer_4k", "tc_prep"): 50.92e6 + 15.08e6,
-                   ("kda_8k", "tc_prep"): 336.78e6 + 291.11e6, ("kda_8k", "tc_chain"): 338.73e6 + 56.62e6,
-                   ("gdn_gva_16k", "tc_prep"): 272.71e6 + 487.64e6, ("gdn_gva_16k", "tc_chain"): 612.41e6 + 120.54e6}
-    dom_bytes = kernel_alg_bytes.get(dom, alg_bytes)
-    dom_s = kernel_ms[dom] / 1e3
-    achieved = dom_bytes / dom_s / 1e9
-    t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
-    t_flop = alg_flops / (peaks["bf16_tflops"] * 1e12)
-    path_s = ms_per_step / 1e3
-    nv_plan, conc_plan = ha.ha_la_prefill_launch_plan(sets[0][0])
-    launch_mode = ("fp32 CUDA-core kernel" if nv_plan == 0 else
-                   f"{nv_plan}-channel slices, prep and chain kernels " + ("side by side" if conc_plan else "back to back"))
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic.get((w.name, dom)),
-                "kernel_alg_bytes": dom_bytes, "peak_source": peaks["source"],
-                "kernel_ms": kernel_ms,      # each kernel alone (sequential launches with events in between)
-                # what the timed steps used (kernel_ms is always back to back, and then with the planner's
-                # back-to-back slice width, which may differ)
-                "launch_mode": launch_mode,
-                "path": {"bound": "hbm" if t_hbm >= t_flop else "tensor", "roofline_us": 1e6 * max(t_hbm, t_flop),
-                         "measured_us": 1e6 * path_s, "frac": max(t_hbm, t_flop) / path_s,
-                         "achieved_gbs": alg_bytes / path_s / 1e9, "achieved_tflops": alg_flops / path_s / 1e12,
-                         "alg_bytes": alg_bytes, "alg_flops": alg_flops}}
+    # ---- parity of the timed configuration, same run: what the LAST timed step wrote, against the oracle
+    parity = None
+    if rank == 0 and not args.no_parity:
+        parity = parity_of(helpers, inp, m["last_out"])
 
     # ---- end to end: pinned host buffers in, o and hT back out, through the public API
     host = {k: (v.cpu().pin_memory() if hasattr(v, "cpu") else v) for k, v in base.items()}
@@ -564,9 +626,29 @@ def main():
     e1.record(s_out)
     barrier()
     e2e_ms = max_over_ranks(dist, e0.elapsed_time(e1), dev)
+    m["check_status"]("during the end-to-end steps")
     e2e = {"value": job_throughput(world, T, e2e_ms / args.steps), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": int(d2h),
            "mode": "two buffer sets, copies of neighbouring steps overlap the compute (3 streams)"}
+
+    # ---- the other full-size workloads, device time only (a few seconds in total): extra rows, not the metric
+    others = None
+    if rank == 0 and world == 1 and not args.no_other_workloads and w.name == "gdn_layer_4k":
+        others = {}
+        del sets, base, m["sets"], m["base"]
+        torch.cuda.empty_cache()
+        for name in ("gdn_gva_16k", "kda_8k", "gdn_varlen"):
+            wo = synth.WORKLOADS[name]
+            io = synth.make_inputs(wo)
+            mo = measure(ha, helpers, wo, io, 30, 5, dev, local_rank, None, peaks, 1)
+            po = parity_of(helpers, io, mo["last_out"]) if not args.no_parity else None
+            others[name] = {"ms_per_step": mo["ms_per_step"], "ms_median": mo["ms_median"], "ms_min": mo["ms_min"],
+                            "tokens_per_s": mo["value"], "steps": 30, "path_frac": mo["roofline"]["path"]["frac"],
+                            "roofline_us": mo["roofline"]["path"]["roofline_us"],
+                            "kernel_ms": mo["roofline"]["kernel_ms"], "launch_mode": mo["roofline"]["launch_mode"],
+                            "clocks": mo["clocks"], "parity": po, "tokens": io["T"]}
+            del mo, io
+            torch.cuda.empty_cache()
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -574,20 +656,26 @@ def main():
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "ms_per_step_median": m["ms_median"],
+                "ms_per_step_min": m["ms_min"], "ms_per_step_max": m["ms_max"], "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
                 "data": "synthetic",
                 "config": {"workload": w.name, "variant": w.variant, "tokens_per_step_per_gpu": T, "sequences": N,
                            "seq_lens": inp["seq_lens"] if N <= 16 else None, "qk_heads": w.hk, "v_heads": w.hv,
-                           "d_k": w.dk, "d_v": w.dv, "chunk": 64, "path": path,
+                           "d_k": w.dk, "d_v": w.dv, "chunk": 64, "path": m["path"],
                            "l2": f"{R} resident input/output sets visited round-robin ({R * alg_bytes / 1e6:.0f} MB), one scratch workspace"
-                                 + (" + L2 flush write between steps" if flush is not None else ""),
+                                 + (" + L2 flush write between steps" if m["flushed"] else ""),
                            "parallelism": "replicas (independent batch per GPU, no collective)" if world > 1 else "1 GPU"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-                "roofline": roofline, "cpu_baseline": cpu, "wall_s_timed_region": t_wall}
+                "clocks": clocks, "e2e": e2e, "gpu_launches": m["launches_per_step"] * args.steps,
+                "roofline": roofline, "parity": parity, "cpu_baseline": cpu, "other_workloads": others,
+                "wall_s_timed_region": m["wall_s"]}
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+    if parity is not None and not parity["ok"]:
+        raise SystemExit(f"parity of the timed configuration failed: {parity}")
+    if others and any(v["parity"] is not None and not v["parity"]["ok"] for v in others.values()):
+        raise SystemExit("parity of another workload failed (see other_workloads in the line above)")
 
 
 if __name__ == "__main__":

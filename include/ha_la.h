@@ -209,6 +209,16 @@ typedef struct {
  * kernel (none when N == 0).                                                                      */
 int ha_la_decode(const ha_la_decode_args* args, void* cuda_stream);
 
+/* Test hook for the device-side bounded waits (the paper has no counterpart).  Every wait inside the
+ * kernels -- on an mbarrier, on another kernel's "chunk is ready" flag -- gives up after a fixed number
+ * of polls, records HA_LA_ERR_TIMEOUT in *status_word and lets the kernel run to a normal exit with
+ * unspecified outputs.  This call makes such a wait run out on purpose, without faulting or hanging
+ * anything: it enqueues ONLY the sequential (state-passing) kernel, in the mode in which it waits per
+ * chunk for the chunk-local kernel's flags, with a flag value that nothing publishes and `spin_limit`
+ * (1 .. 2^20) polls per wait.  Arguments as for ha_la_prefill (bf16, d = 128, equal-length rows,
+ * status_word required); o and hT receive meaningless numbers.  Returns HA_LA_OK once enqueued.       */
+int ha_la_debug_wait_timeout(const ha_la_prefill_args* args, void* cuda_stream, unsigned int spin_limit);
+
 const char* ha_la_status_string(int status);
 int ha_la_version(void);
 

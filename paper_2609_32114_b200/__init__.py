@@ -7,6 +7,7 @@ library has not been built.
 """
 from .binding import (  # noqa: F401
     HaLaError,
+    ha_la_debug_wait_timeout,
     ha_la_decode,
     ha_la_decode_args,
     ha_la_decode_raw,

@@ -33,6 +33,7 @@ EXPORTS = (
     "ha_la_prefill_num_launches",
     "ha_la_prefill_launch_plan",
     "ha_la_decode",
+    "ha_la_debug_wait_timeout",
     "ha_la_status_string",
     "ha_la_version",
 )
@@ -128,6 +129,8 @@ def load_library(path: Optional[str] = None):
     lib.ha_la_prefill_launch_plan.restype = ctypes.c_int
     lib.ha_la_decode.argtypes = [ctypes.POINTER(ha_la_decode_args), ctypes.c_void_p]
     lib.ha_la_decode.restype = ctypes.c_int
+    lib.ha_la_debug_wait_timeout.argtypes = [A, ctypes.c_void_p, ctypes.c_uint]
+    lib.ha_la_debug_wait_timeout.restype = ctypes.c_int
     lib.ha_la_status_string.argtypes = [ctypes.c_int]
     lib.ha_la_status_string.restype = ctypes.c_char_p
     lib.ha_la_version.argtypes = []
@@ -192,6 +195,12 @@ def ha_la_prefill_noalloc(args: ha_la_prefill_args, stream: int = 0) -> int:
     """The C call for callers that cannot supply scratch memory (the workspace fields are ignored);
     returns the status code.  See include/ha_la.h for its limits and its sharing rules."""
     return load_library().ha_la_prefill_noalloc(ctypes.byref(args), ctypes.c_void_p(stream) if stream else None)
+
+
+def ha_la_debug_wait_timeout(args: ha_la_prefill_args, stream: int = 0, spin_limit: int = 4096) -> int:
+    """Test hook: the sequential kernel alone, waiting for flags nothing publishes; returns the status code."""
+    return load_library().ha_la_debug_wait_timeout(ctypes.byref(args), ctypes.c_void_p(stream) if stream else None,
+                                                   ctypes.c_uint(spin_limit))
 
 
 def ha_la_prefill_noalloc_scratch_bytes() -> int:

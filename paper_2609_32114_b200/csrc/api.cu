@@ -174,6 +174,22 @@ int ha_la_prefill_timed(const ha_la_prefill_args* a, void* cuda_stream, int max_
   return rc;
 }
 
+int ha_la_debug_wait_timeout(const ha_la_prefill_args* a, void* cuda_stream, unsigned int spin_limit) {
+  Problem p;
+  int rc = make_problem(a, &p);
+  if (rc != HA_LA_OK) return rc;
+  if (!tc_supported(p) || a->cu_seqlens || a->num_seqs > 0) return HA_LA_ERR_UNSUPPORTED;
+  if (!a->q || !a->k || !a->v || !a->g || !a->beta || !a->o || !a->status_word) return HA_LA_ERR_INVALID_ARG;
+  if (spin_limit < 1 || spin_limit > (1u << 20)) return HA_LA_ERR_INVALID_ARG;
+  size_t need = 0;
+  rc = ha_la_prefill_workspace_bytes(a, &need);
+  if (rc != HA_LA_OK) return rc;
+  if (!a->workspace || ((uintptr_t)a->workspace & 255) || a->workspace_bytes < need) return HA_LA_ERR_WORKSPACE;
+  void* tc_ws = reinterpret_cast<char*>(a->workspace) + plan_bytes(p);
+  return launch_tc_chain_unpublished(p, *a, tc_ws, spin_limit, reinterpret_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? HA_LA_OK : HA_LA_ERR_CUDA;
+}
+
 const char* ha_la_status_string(int status) {
   switch (status) {
     case HA_LA_OK: return "ok";

@@ -71,6 +71,8 @@ int tc_num_launches(const Problem& p);
 void tc_launch_plan(const Problem& p, int* slice_width, int* concurrent);   // what launch_tc would choose
 cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView plan, void* tc_ws,
                       cudaStream_t stream);
+cudaError_t launch_tc_chain_unpublished(const Problem& p, const ha_la_prefill_args& a, void* tc_ws, uint32_t spin_limit,
+                                        cudaStream_t stream);
 
 // Optional per-kernel event timing (ha_la_prefill_timed): every launcher marks the stream before its kernel.
 struct KernelTimer {

@@ -15,6 +15,11 @@
     if (threadIdx.x == 0 && blockIdx.x == 0 && (slot) < 1024) g_prof_##name[slot] = clock64(); \
   } while (0)
 #endif
+// the same for a thread of the caller's choice (CTA 0 only)
+#define HA_PROF_ANY(name, slot)                                                        \
+  do {                                                                                 \
+    if (blockIdx.x == 0 && (slot) < 1024) g_prof_##name[slot] = clock64();             \
+  } while (0)
 // records the SM id of CTA `blockIdx.x` at slot base + blockIdx.x % count
 #define HA_PROF_SMID(name, base, count)                                                \
   do {                                                                                 \
@@ -33,6 +38,7 @@
   } while (0)
 #else
 #define HA_PROF_GT(name, slot) do { } while (0)
+#define HA_PROF_ANY(name, slot) do { } while (0)
 #define HA_PROF_SMID(name, base, count) do { } while (0)
 #define HA_PROF_DECL(name)
 #define HA_PROF(name, slot) do { } while (0)

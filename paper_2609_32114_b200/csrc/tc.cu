@@ -25,7 +25,7 @@ cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanVi
                            int reserved_sms, cudaStream_t stream);
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                             const CUtensorMap& mk, const CUtensorMap& mo, int nv, int64_t epoch, bool dependent,
-                            cudaStream_t stream);
+                            uint32_t spin_limit, cudaStream_t stream);
 
 cudaError_t configure_tc_prep(const Problem& p);
 cudaError_t configure_tc_chain(const Problem& p, int nv);
@@ -86,6 +86,7 @@ int sm_count() {
 }
 
 constexpr int kMaxDevices = 64;
+constexpr uint32_t kDefaultSpinLimit = 4u << 20;      // polls before a device-side bounded wait gives up
 std::atomic<uint32_t> g_calls{0};
 
 // Epoch of a concurrent-mode call: (random per-process tag, never 0) << 32 | call counter.
@@ -219,7 +220,21 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   }
   cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, reserved_sms, stream);
   if (e != cudaSuccess) return e;
-  return launch_tc_chain(p, a, plan, ws, mk, mo, nv, epoch, /*dependent=*/g_timer == nullptr, stream);
+  return launch_tc_chain(p, a, plan, ws, mk, mo, nv, epoch, /*dependent=*/g_timer == nullptr, kDefaultSpinLimit, stream);
+}
+
+// Test hook behind ha_la_debug_wait_timeout: the sequential kernel alone, in the concurrent mode, with an epoch that
+// nothing will ever publish and a small poll limit.  Its first flag wait runs out, it records the time-out, and then
+// walks the chunks on whatever the workspace holds (valid memory, meaningless numbers) to a normal exit.
+cudaError_t launch_tc_chain_unpublished(const Problem& p, const ha_la_prefill_args& a, void* tc_ws, uint32_t spin_limit,
+                                        cudaStream_t stream) {
+  const int nv = 32;
+  CUtensorMap mk, mo;
+  if (!make_map(&mk, a.k, p.T_total, p.HK) || !make_map_o(&mo, a.o, p.T_total, p.HV, nv)) return cudaErrorInvalidValue;
+  const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
+  cudaError_t ce = configure_tc_chain(p, nv);
+  if (ce != cudaSuccess) return ce;
+  return launch_tc_chain(p, a, PlanView{}, ws, mk, mo, nv, next_epoch(), /*dependent=*/false, spin_limit, stream);
 }
 
 }  // namespace ha_la

@@ -74,6 +74,7 @@ struct ChainParams {
   float scale;
   int64_t epoch;               // != 0: the prep kernel runs concurrently; wait for ws.flags[cj] == epoch per chunk
                                // == 0: wait for the whole prep grid before the first workspace read
+  uint32_t spin_limit;         // polls before a bounded wait gives up (kSpinLimit; a few thousand in the time-out test)
   int32_t* status;
 };
 
@@ -207,7 +208,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
     for (int c = 0; c < nchunks; ++c) {
       if (c >= ready_upto) {
         int got = 0;
-        for (uint32_t it = 0; it < kSpinLimit && !*abort_flag; ++it) {
+        for (uint32_t it = 0; it < p.spin_limit && !*abort_flag; ++it) {
           const int cc = c + lane;
           bool ok = false;
           if (cc < nchunks)
@@ -226,7 +227,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
       }
       if (lane == 0) {
         const int st = c % S;
-        if (c >= S) mbar_wait(&bar_empty[st], ((c / S) - 1) & 1, abort_flag);
+        if (c >= S) mbar_wait(&bar_empty[st], ((c / S) - 1) & 1, abort_flag, p.spin_limit);
         uint8_t* stage = sm + st * Cfg::kStageB;
         const size_t cj = (size_t)(chunk0 + c) * p.HV + j;
         mbar_expect_tx(&bar_full[st], Cfg::kTxBytes);
@@ -254,7 +255,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
       const uint32_t stage = smem_u32(sm + st * Cfg::kStageB);
       const uint64_t dWQ = smem_desc(stage + Cfg::OFF_WQ, 16384, 1024, kSwizzle128B);
       const uint64_t dK = smem_desc(stage + Cfg::OFF_K, 8192, 1024, kSwizzle128B);
-      if (lead) mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
+      if (lead) mbar_wait(&bar_full[st], (c / S) & 1, abort_flag, p.spin_limit);
       named_sync(BAR_H_READY, NCOMP + 32);               // h (bf16) of the previous chunk is in sH
       if (lead) {
         tc_fence_after_sync();
@@ -306,7 +307,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
       const uint32_t ph = c & 1;
 
       HA_PROF(chain, 8 * c + 0);
-      mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
+      mbar_wait(&bar_full[st], (c / S) & 1, abort_flag, p.spin_limit);
       HA_PROF(chain, 8 * c + 1);
       // operands of the first epilogue that do not depend on the MMA, fetched while it runs
       const float* sc = reinterpret_cast<const float*>(stage + Cfg::OFF_SC);
@@ -315,7 +316,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
       float pre[32];
       load_img32(stage + (row < 64 ? Cfg::OFF_U : Cfg::OFF_O), i, cg0, pre);
 
-      mbar_wait(bar_mma1, ph, abort_flag);
+      mbar_wait(bar_mma1, ph, abort_flag, p.spin_limit);
       HA_PROF(chain, 8 * c + 2);
       tc_fence_after_sync();
       if (row < 64) {                                    // U~ rows: (U - W h) e^{G_L - G_i}, the MMA2 operand
@@ -375,7 +376,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
         }
       }
 
-      mbar_wait(bar_mma2, ph, abort_flag);
+      mbar_wait(bar_mma2, ph, abort_flag, p.spin_limit);
       HA_PROF(chain, 8 * c + 4);
       tc_fence_after_sync();
       mbar_arrive(&bar_empty[st]);                       // this thread and both MMAs are done with the stage
@@ -506,7 +507,7 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     for (int c = 0; c < nchunks; ++c) {
       if (c >= ready_upto) {
         int got = 0;
-        for (uint32_t it = 0; it < kSpinLimit && !*abort_flag; ++it) {
+        for (uint32_t it = 0; it < p.spin_limit && !*abort_flag; ++it) {
           const int cc = c + lane;
           bool ok = false;
           if (cc < nchunks)
@@ -524,7 +525,7 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       }
       if (lane == 0) {
         const int st = c % S;
-        if (c >= S) mbar_wait(&bar_empty[st], ((c / S) - 1) & 1, abort_flag);
+        if (c >= S) mbar_wait(&bar_empty[st], ((c / S) - 1) & 1, abort_flag, p.spin_limit);
         uint8_t* stage = sm + st * Cfg::kStageB;
         const size_t cj = (size_t)(chunk0 + c) * p.HV + j;
         mbar_expect_tx(&bar_full[st], Cfg::kTxBytes);
@@ -553,7 +554,7 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       const uint64_t dWQ = smem_desc(stage + Cfg::OFF_WQ, 16384, 1024, kSwizzle128B);   // N = 64 W + 64 Q~ tokens
       const uint64_t dK = smem_desc(stage + Cfg::OFF_K, 8192, 1024, kSwizzle128B);      // N = 2 x 64 key channels
       const uint32_t d1 = tmem + Cfg::TM_D1 + (c & 1) * 128;
-      if (lead) mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
+      if (lead) mbar_wait(&bar_full[st], (c / S) & 1, abort_flag, p.spin_limit);
       named_sync(BAR_H_READY, NCOMP + 32);               // h^T (bf16 pairs) of the previous chunk is in tensor memory
       if (lead) {
         tc_fence_after_sync();
@@ -664,12 +665,12 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       const uint8_t* stage = sm + st * Cfg::kStageB;
       const uint32_t ph = c & 1;
       HA_PROF(chain, 8 * c + 0);
-      mbar_wait(&bar_full[st], (c / S) & 1, abort_flag);
+      mbar_wait(&bar_full[st], (c / S) & 1, abort_flag, p.spin_limit);
       HA_PROF(chain, 8 * c + 1);
       const float* sc = reinterpret_cast<const float*>(stage + Cfg::OFF_SC);
       float u[TOK];                                      // U^T[v][TOK g ..], fetched while MMA1 runs
       img_row(stage + Cfg::OFF_U, u);
-      mbar_wait(bar_mma1, ph, abort_flag);
+      mbar_wait(bar_mma1, ph, abort_flag, p.spin_limit);
       HA_PROF(chain, 8 * c + 2);
       tc_fence_after_sync();
       {
@@ -689,7 +690,7 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       named_arrive(BAR_U_READY, NCOMP + 32);
       HA_PROF(chain, 8 * c + 3);
 
-      mbar_wait(bar_mma2, ph, abort_flag);
+      mbar_wait(bar_mma2, ph, abort_flag, p.spin_limit);
       HA_PROF(chain, 8 * c + 4);
       tc_fence_after_sync();
 #pragma unroll
@@ -801,7 +802,7 @@ cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, const CUte
 
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                             const CUtensorMap& mk, const CUtensorMap& mo, int nv, int64_t epoch, bool dependent,
-                            cudaStream_t stream) {
+                            uint32_t spin_limit, cudaStream_t stream) {
   ChainParams cp;
   cp.h0 = a.h0; cp.hT = a.hT; cp.o = a.o;
   cp.seq_tok0 = plan.seq_tok0; cp.seq_len = plan.seq_len; cp.seq_chunk0 = plan.seq_chunk0;
@@ -809,6 +810,7 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   cp.T_row = p.T_row; cp.cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
   cp.ws = ws; cp.HK = p.HK; cp.HV = p.HV; cp.scale = p.scale; cp.status = a.status_word;
   cp.epoch = epoch;
+  cp.spin_limit = spin_limit;
   const int grid = p.N * p.HV * (128 / nv);
   if (grid == 0) return cudaSuccess;
   return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, &mo, nv, grid, dependent, stream)

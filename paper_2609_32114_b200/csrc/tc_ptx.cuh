@@ -37,10 +37,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Non-blocking test (try_wait may suspend the thread for a system-dependent time): for loops that poll several
+// barriers at once.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+
 // Bounded wait.  Gives up after `kSpinLimit` polls (or at once when *abort is already set), sets
 // *abort and returns false; the caller carries on with the same control flow (results are then
 // unspecified and the status word reports HA_LA_ERR_TIMEOUT), so no barrier count ever diverges.
+#ifdef HA_EXP_SPIN
+constexpr uint32_t kSpinLimit = HA_EXP_SPIN;   // (developer experiments: give up quickly)
+#else
 constexpr uint32_t kSpinLimit = 4u << 20;
+#endif
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort,
                                           uint32_t limit = kSpinLimit) {
   for (uint32_t it = 0; it < limit; ++it) {

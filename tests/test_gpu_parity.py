@@ -179,6 +179,26 @@ def test_bad_cu_seqlens_reports_device_check():
     torch.cuda.synchronize()
 
 
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """Every device-side wait is bounded.  The test hook launches the sequential kernel alone, waiting per chunk for
+    flags that nothing publishes, with a limit of a few thousand polls: the wait must run out, the status word must
+    say HA_LA_ERR_TIMEOUT, the kernel must exit normally, and the library must work as before afterwards."""
+    import torch
+    import paper_2609_32114_b200 as ha
+    from paper_2609_32114_b200 import binding
+
+    w = synth.shrink(W["gdn_layer_4k"], seq_lens=[300], hk=1, hv=2)
+    inp = synth.make_inputs(w, seed=83)
+    d = helpers.to_device(inp)
+    args, keep = ha.prepare_args(d["q"], d["k"], d["v"], d["g"], d["beta"], variant="gdn")
+    keep["workspace"].zero_()
+    rc = ha.ha_la_debug_wait_timeout(args, torch.cuda.current_stream().cuda_stream, 3000)
+    assert rc == 0, ha.status_string(rc)
+    torch.cuda.synchronize()                                   # returns: nothing hangs, nothing faults
+    assert int(keep["status_word"].item()) == binding.HA_LA_ERR_TIMEOUT
+    helpers.check_parity(inp)                                  # the next ordinary call is unaffected
+
+
 # ---------------------------------------------------------------- full-size configurations, every head
 
 @pytest.mark.parametrize("name", ["gdn_layer_4k", "gdn_gva_16k", "kda_8k", "gdn_varlen"])
