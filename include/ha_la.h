@@ -141,6 +141,14 @@ int ha_la_prefill_num_launches(const ha_la_prefill_args* args);
  * Returns HA_LA_OK, or an error for invalid / unsupported shapes or NULL outputs.               */
 int ha_la_prefill_launch_plan(const ha_la_prefill_args* args, int* slice_width, int* concurrent);
 
+/* Segments per sequence ha_la_prefill would use for these shapes (host only; 1 = the chunks of a sequence are
+ * walked strictly in order; 0 if the shapes are unsupported).  With S > 1 a sequence's chunks are cut into S
+ * runs that are walked at the same time -- the Chunk-Seg-Seg mapping the paper describes for its FlashQLA
+ * baseline (Section 4.1): later segments start from a zero state and from the identity, and their true start
+ * states, final state and outputs follow from one affine fix-up per segment.  Chosen only for equal-length rows
+ * with so few (sequence, head) pairs that every run still gets an SM; HA_LA_TC_SEGMENTS overrides it.            */
+int ha_la_prefill_num_segments(const ha_la_prefill_args* args);
+
 /* Profiling aid (the paper's "Metrics" paragraph times kernels with device events): the same work
  * as ha_la_prefill, with a CUDA event recorded on `cuda_stream` before every kernel and after the
  * last one.  Unlike ha_la_prefill it BLOCKS until the stream has drained, then writes the device

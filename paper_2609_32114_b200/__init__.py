@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     ha_la_prefill_args,
     ha_la_prefill_launch_plan,
     ha_la_prefill_num_launches,
+    ha_la_prefill_num_segments,
     ha_la_prefill_path,
     ha_la_prefill_noalloc,
     ha_la_prefill_noalloc_scratch_bytes,

@@ -32,6 +32,7 @@ EXPORTS = (
     "ha_la_prefill_path",
     "ha_la_prefill_num_launches",
     "ha_la_prefill_launch_plan",
+    "ha_la_prefill_num_segments",
     "ha_la_decode",
     "ha_la_debug_wait_timeout",
     "ha_la_status_string",
@@ -125,6 +126,8 @@ def load_library(path: Optional[str] = None):
     lib.ha_la_prefill_path.restype = ctypes.c_char_p
     lib.ha_la_prefill_num_launches.argtypes = [A]
     lib.ha_la_prefill_num_launches.restype = ctypes.c_int
+    lib.ha_la_prefill_num_segments.argtypes = [A]
+    lib.ha_la_prefill_num_segments.restype = ctypes.c_int
     lib.ha_la_prefill_launch_plan.argtypes = [A, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
     lib.ha_la_prefill_launch_plan.restype = ctypes.c_int
     lib.ha_la_decode.argtypes = [ctypes.POINTER(ha_la_decode_args), ctypes.c_void_p]
@@ -175,6 +178,11 @@ def ha_la_prefill_path(args: ha_la_prefill_args) -> Optional[str]:
 
 def ha_la_prefill_num_launches(args: ha_la_prefill_args) -> int:
     return load_library().ha_la_prefill_num_launches(ctypes.byref(args))
+
+
+def ha_la_prefill_num_segments(args: ha_la_prefill_args) -> int:
+    """Segments a sequence's chunks are cut into (1 = walked strictly in order)."""
+    return load_library().ha_la_prefill_num_segments(ctypes.byref(args))
 
 
 def ha_la_prefill_launch_plan(args: ha_la_prefill_args) -> Tuple[int, bool]:

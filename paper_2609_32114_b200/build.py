@@ -20,7 +20,7 @@ LIB = os.path.join(PKG, "libha_la.so")
 INCLUDE = os.path.join(ROOT, "include")
 
 # (object name, source, extra flags)
-UNITS = [("api", "api.cu", []), ("plan", "plan.cu", []), ("tc", "tc.cu", []), ("tc_prep", "tc_prep.cu", []), ("tc_chain", "tc_chain.cu", []),
+UNITS = [("api", "api.cu", []), ("plan", "plan.cu", []), ("tc", "tc.cu", []), ("tc_prep", "tc_prep.cu", []), ("tc_chain", "tc_chain.cu", []), ("tc_seg", "tc_seg.cu", []),
          ("noalloc", "noalloc.cu", []), ("decode", "decode.cu", [])] + [
     (f"simt{u}", "simt.cu", [f"-DHA_LA_SIMT_UNIT={u}"]) for u in range(5)
 ]

@@ -43,6 +43,7 @@ int make_problem(const ha_la_prefill_args* a, Problem* p) {
   p->dk = a->d_k;
   p->dv = a->d_v;
   p->scale = a->scale;
+  p->varlen = varlen ? 1 : 0;
   if (varlen) {
     p->max_len = (a->max_seqlen > 0 && a->max_seqlen < a->seqlen) ? a->max_seqlen : a->seqlen;
     p->max_chunks = (int)(((long long)p->T_total + 63LL * p->N) / kChunk);
@@ -94,6 +95,12 @@ int ha_la_prefill_num_launches(const ha_la_prefill_args* args) {
   Problem p;
   if (make_problem(args, &p) != HA_LA_OK) return 0;
   return (needs_plan(args, p) ? 1 : 0) + (use_tc(p) ? tc_num_launches(p) : 1);
+}
+
+int ha_la_prefill_num_segments(const ha_la_prefill_args* args) {
+  Problem p;
+  if (make_problem(args, &p) != HA_LA_OK) return 0;
+  return use_tc(p) ? tc_num_segments(p) : 1;
 }
 
 int ha_la_prefill_launch_plan(const ha_la_prefill_args* args, int* slice_width, int* concurrent) {

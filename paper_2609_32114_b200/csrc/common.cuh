@@ -35,6 +35,7 @@ struct Problem {
   int max_chunks;   // bound on chunk slots (MC)
   int max_seq_chunks;
   float scale;
+  int varlen;       // packed batch (cu_seqlens) rather than equal-length rows
 };
 
 inline __host__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -68,6 +69,7 @@ bool simt_supported(const Problem& p);
 bool tc_supported(const Problem& p);
 size_t tc_workspace_bytes(const Problem& p);
 int tc_num_launches(const Problem& p);
+int tc_num_segments(const Problem& p);                                      // segments per sequence launch_tc would use
 void tc_launch_plan(const Problem& p, int* slice_width, int* concurrent);   // what launch_tc would choose
 cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView plan, void* tc_ws,
                       cudaStream_t stream);

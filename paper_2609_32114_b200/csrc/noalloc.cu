@@ -65,6 +65,7 @@ extern "C" int ha_la_prefill_noalloc(const ha_la_prefill_args* a, void* cuda_str
   p.T_row = a->seqlen;
   p.HK = a->num_qk_heads; p.HV = a->num_v_heads; p.dk = a->d_k; p.dv = a->d_v;
   p.scale = a->scale;
+  p.varlen = packed ? 1 : 0;
   if (packed) {
     p.max_len = (a->max_seqlen > 0 && a->max_seqlen < a->seqlen) ? a->max_seqlen : a->seqlen;
     p.max_chunks = (int)(((long long)p.T_total + 63LL * p.N) / kChunk);

@@ -25,7 +25,8 @@ cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanVi
                            int reserved_sms, cudaStream_t stream);
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                             const CUtensorMap& mk, const CUtensorMap& mo, int nv, int64_t epoch, bool dependent,
-                            uint32_t spin_limit, cudaStream_t stream);
+                            uint32_t spin_limit, const SegBuffers& sg, cudaStream_t stream);
+cudaError_t launch_tc_seg_fix(const Problem& p, const ha_la_prefill_args& a, const SegBuffers& sg, cudaStream_t stream);
 
 cudaError_t configure_tc_prep(const Problem& p);
 cudaError_t configure_tc_chain(const Problem& p, int nv);
@@ -113,7 +114,7 @@ int64_t next_epoch() {
 // interference), plus the wait for the first chunks; with several sequences the prep kernel works through them
 // one after the other, so the last sequence's chain starts only when most of the prep work is done.
 // Only bounds are known on the host: max_len for the longest sequence, max_chunks for the total.
-struct TcPlan { int nv; bool concurrent; };
+struct TcPlan { int nv; bool concurrent; int nseg; };
 
 TcPlan plan_tc(const Problem& p) {
   const int sms = sm_count();
@@ -134,7 +135,7 @@ TcPlan plan_tc(const Problem& p) {
   // cannot be packed any better than in rounds of one CTA per SM
   const double avg_len = p.N > 0 ? (double)p.T_total / p.N : 0.0;
   const bool even = avg_len <= 0.0 || p.max_len < 1.5 * avg_len;
-  bool may_overlap = !g_timer && p.max_chunks > 1;       // (timing wants one kernel at a time)
+  bool may_overlap = p.max_chunks > 1;
   bool force_overlap = false;                            // "2": side by side whenever that is legal (tests)
   if (const char* e = getenv("HA_LA_TC_OVERLAP")) {
     may_overlap = may_overlap && e[0] != '0';
@@ -145,7 +146,7 @@ TcPlan plan_tc(const Problem& p) {
     const int v = atoi(e);
     if (v == 32 || v == 64 || v == 128) forced_nv = v;
   }
-  TcPlan plan{32, false};
+  TcPlan plan{32, false, 1};
   double best = 1e30;
   for (int w = 0; w < 3; ++w) {
     if (forced_nv && widths[w] != forced_nv) continue;
@@ -157,7 +158,7 @@ TcPlan plan_tc(const Problem& p) {
       chain_us = even ? serial * (double)((ctas + sms - 1) / sms) : (serial > spread ? serial : spread);
     }
     const double back_to_back = prep_us + chain_us + (force_overlap ? 1e9 : 0.0);
-    if (back_to_back < best) { best = back_to_back; plan = TcPlan{widths[w], false}; }
+    if (back_to_back < best) { best = back_to_back; plan = TcPlan{widths[w], false, 1}; }
     if (may_overlap && ctas * 2 <= sms) {
       const double prep_beside = 1.1 * prep_time(sms - (int)ctas);
       double overlapped = (chain_us > prep_beside ? chain_us : prep_beside) + 12.0;
@@ -165,7 +166,33 @@ TcPlan plan_tc(const Problem& p) {
         const double last = prep_beside * (1.0 - 1.0 / p.N) + chain_us + 12.0;
         if (last > overlapped) overlapped = last;
       }
-      if (overlapped < best) { best = overlapped; plan = TcPlan{widths[w], true}; }
+      if (overlapped < best) { best = overlapped; plan = TcPlan{widths[w], true, 1}; }
+    }
+  }
+  // Segment-parallel state passing (equal-length rows, sliced kernels, back to back with the prep kernel): a
+  // sequence's chain is cut into nseg segments that run at once; a later segment costs three times the columns of
+  // the first (its own from a zero state plus 128 transition columns), so it only pays while all those CTAs have an
+  // SM each, i.e. for few heads and long sequences.  Costs measured on B200: the chain's per-chunk times above, some
+  // 3 us per segment for the start states and about a quarter of a microsecond of one SM per corrected chunk-head.
+  int forced_seg = 0;
+  if (const char* e = getenv("HA_LA_TC_SEGMENTS")) {
+    const int v = atoi(e);
+    if (v == 1 || v == 2 || v == 4 || v == 8) forced_seg = v;
+  }
+  if (!p.varlen && forced_seg != 1 && longest >= 2) {
+    for (int w = 0; w < 2; ++w) {                          // 32- and 64-channel slices
+      if (forced_nv && widths[w] != forced_nv) continue;
+      for (int nseg = 2; nseg <= 8; nseg *= 2) {
+        if (forced_seg && nseg != forced_seg) continue;
+        if (nseg > longest) continue;
+        const long long ctas = chains * (128 / widths[w]) * (2 * nseg - 1);
+        if (ctas > sms && !forced_seg) continue;
+        const double cpseg = (double)(long long)((longest + nseg - 1) / nseg);
+        const double waves = (double)((ctas + sms - 1) / sms);
+        const double later = items * (1.0 - 1.0 / nseg);
+        const double t = prep_us + waves * cpseg * per_chunk_us[w] + 4.0 + 3.0 * (nseg - 1) + 5.0 + later * 0.25 / sms;
+        if (t < best || (forced_seg && plan.nseg != forced_seg)) { best = t; plan = TcPlan{widths[w], false, nseg}; }
+      }
     }
   }
   return plan;
@@ -177,11 +204,16 @@ bool tc_supported(const Problem& p) {
   return p.dtype == HA_LA_BF16 && p.dk == 128 && p.dv == 128;
 }
 
+// (the largest segment count the planner may pick, so that the environment switches cannot outgrow a workspace
+// that was sized before they were set)
 size_t tc_workspace_bytes(const Problem& p) {
-  return tc_ws_bytes_for((size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
+  const size_t img = tc_ws_bytes_for((size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
+  return img + (p.varlen ? 0 : tc_seg_bytes((size_t)p.N * p.HV, 8, (size_t)p.T_total, p.HV));
 }
 
-int tc_num_launches(const Problem&) { return 2; }
+int tc_num_launches(const Problem& p) { return plan_tc(p).nseg > 1 ? 4 : 2; }
+
+int tc_num_segments(const Problem& p) { return plan_tc(p).nseg; }
 
 void tc_launch_plan(const Problem& p, int* slice_width, int* concurrent) {
   const TcPlan tp = plan_tc(p);
@@ -196,8 +228,11 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   if (!make_map(&mq, a.q, p.T_total, p.HK) || !make_map(&mk, a.k, p.T_total, p.HK) ||
       !make_map(&mv, a.v, p.T_total, p.HV) || !make_map_o(&mo, a.o, p.T_total, p.HV, nv))
     return cudaErrorInvalidValue;
-  const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
-  const bool concurrent = tp.concurrent;
+  const size_t ncj = (size_t)p.max_chunks * p.HV;
+  const TcWorkspace ws = tc_ws_view(tc_ws, ncj, p.variant == HA_LA_KDA);
+  const SegBuffers sg = tc_seg_view(reinterpret_cast<uint8_t*>(tc_ws) + tc_ws_bytes_for(ncj, p.variant == HA_LA_KDA),
+                                    (size_t)p.N * p.HV, tp.nseg, (size_t)p.T_total, p.HV);
+  const bool concurrent = tp.concurrent && !g_timer;     // (per-kernel timing wants one kernel at a time)
   // Configure (and load) both kernels before anything is enqueued: loading a kernel for the first time can
   // wait for the device, and in the concurrent mode the chain kernel would be spinning meanwhile.
   // (Once per device and kernel instance: the attributes stick, and the calls are not free on the host.)
@@ -220,7 +255,9 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   }
   cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, reserved_sms, stream);
   if (e != cudaSuccess) return e;
-  return launch_tc_chain(p, a, plan, ws, mk, mo, nv, epoch, /*dependent=*/g_timer == nullptr, kDefaultSpinLimit, stream);
+  e = launch_tc_chain(p, a, plan, ws, mk, mo, nv, epoch, /*dependent=*/g_timer == nullptr, kDefaultSpinLimit, sg, stream);
+  if (e != cudaSuccess) return e;
+  return launch_tc_seg_fix(p, a, sg, stream);
 }
 
 // Test hook behind ha_la_debug_wait_timeout: the sequential kernel alone, in the concurrent mode, with an epoch that
@@ -234,7 +271,8 @@ cudaError_t launch_tc_chain_unpublished(const Problem& p, const ha_la_prefill_ar
   const TcWorkspace ws = tc_ws_view(tc_ws, (size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
   cudaError_t ce = configure_tc_chain(p, nv);
   if (ce != cudaSuccess) return ce;
-  return launch_tc_chain(p, a, PlanView{}, ws, mk, mo, nv, next_epoch(), /*dependent=*/false, spin_limit, stream);
+  return launch_tc_chain(p, a, PlanView{}, ws, mk, mo, nv, next_epoch(), /*dependent=*/false, spin_limit,
+                         SegBuffers{1, nullptr, nullptr, nullptr, nullptr}, stream);
 }
 
 }  // namespace ha_la

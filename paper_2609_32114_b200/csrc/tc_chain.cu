@@ -75,6 +75,15 @@ struct ChainParams {
   int64_t epoch;               // != 0: the prep kernel runs concurrently; wait for ws.flags[cj] == epoch per chunk
                                // == 0: wait for the whole prep grid before the first workspace read
   uint32_t spin_limit;         // polls before a bounded wait gives up (kSpinLimit; a few thousand in the time-out test)
+  // Segment-parallel state passing (sliced kernels, equal-length rows): a sequence's chunks are cut into `nseg`
+  // segments that run at the same time.  Segment 0 starts from h0.  A later segment s runs twice over: its value
+  // columns from a ZERO state (provisional outputs into o, end state b_s into seg_b) and 128 "transition" columns
+  // from the IDENTITY with U = O_loc = 0 (end state Phi_s into seg_phi; its output rows are R = scale Q~ Phi,
+  // written to r_out).  The true start state h_s of the segment then gives  o += R h_s  and  h_{s+1} = Phi_s h_s + b_s.
+  int nseg;                    // 1: off
+  float* seg_b;                // [N*HV][nseg][128][128] fp32
+  float* seg_phi;              // [N*HV][nseg][128][128] fp32
+  void* r_out;                 // [T][HV][128], dtype of o
   int32_t* status;
 };
 
@@ -166,13 +175,24 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
   const int slice = blockIdx.x % NSL;
-  const int nj = blockIdx.x / NSL;
+  const int unit_id = blockIdx.x / NSL;
+  const int units = 2 * p.nseg - 1;                      // per (sequence, V-head): nseg value runs + (nseg - 1) transition runs
+  const int unit = unit_id % units;
+  const int nj = unit_id / units;
+  const int seg = unit < p.nseg ? unit : unit - p.nseg + 1;
+  const bool trans = unit >= p.nseg;                     // this CTA carries transition columns (see ChainParams)
   const int j = nj % p.HV;
   const int n = p.seq_order ? p.seq_order[nj / p.HV] : nj / p.HV;   // CTAs of the longest sequences come first
   const int jq = j / (p.HV / p.HK);
-  const int tok0 = p.seq_tok0 ? p.seq_tok0[n] : n * p.T_row;
-  const int len = p.seq_tok0 ? p.seq_len[n] : p.T_row;
-  const int chunk0 = p.seq_tok0 ? p.seq_chunk0[n] : n * p.cps;
+  const int tok0_seq = p.seq_tok0 ? p.seq_tok0[n] : n * p.T_row;
+  const int len_seq = p.seq_tok0 ? p.seq_len[n] : p.T_row;
+  const int chunk0_seq = p.seq_tok0 ? p.seq_chunk0[n] : n * p.cps;
+  // this CTA's segment of the sequence, walked like a sequence of its own
+  const int nch_seq = (len_seq + kChunk - 1) / kChunk;
+  const int cpseg = (nch_seq + p.nseg - 1) / p.nseg;
+  const int tok0 = tok0_seq + seg * cpseg * kChunk;
+  const int len = max(0, min(len_seq - seg * cpseg * kChunk, cpseg * kChunk));
+  const int chunk0 = chunk0_seq + seg * cpseg;
   const int nchunks = (len + kChunk - 1) / kChunk;
 
   if (blockIdx.x == 0 && threadIdx.x == 0) HA_PROF_GT(chain, 900);
@@ -230,10 +250,12 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
         if (c >= S) mbar_wait(&bar_empty[st], ((c / S) - 1) & 1, abort_flag, p.spin_limit);
         uint8_t* stage = sm + st * Cfg::kStageB;
         const size_t cj = (size_t)(chunk0 + c) * p.HV + j;
-        mbar_expect_tx(&bar_full[st], Cfg::kTxBytes);
+        mbar_expect_tx(&bar_full[st], Cfg::kTxBytes - (trans ? 2 * Cfg::kSliceB : 0));
         bulk_load(stage + Cfg::OFF_WQ, p.ws.wq + cj * 2 * kImgBytes, 32768, &bar_full[st]);
-        bulk_load(stage + Cfg::OFF_U, p.ws.u + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
-        bulk_load(stage + Cfg::OFF_O, p.ws.ol + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
+        if (!trans) {                                    // (transition columns: U = O_loc = 0)
+          bulk_load(stage + Cfg::OFF_U, p.ws.u + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
+          bulk_load(stage + Cfg::OFF_O, p.ws.ol + cj * kImgBytes + (size_t)slice * Cfg::kSliceB, Cfg::kSliceB, &bar_full[st]);
+        }
         bulk_load(stage + Cfg::OFF_SC, p.ws.sc + cj * kScFloats, 768, &bar_full[st]);
         if constexpr (KDA) {   // K e^{G_L - G} from the prep kernel (per-channel decay cannot be applied to U~ rows)
           bulk_load(stage + Cfg::OFF_K, p.ws.kd + cj * kImgBytes, 16384, &bar_full[st]);
@@ -284,8 +306,12 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
 #pragma unroll
       for (int q = 0; q < NVT; q += 4) {
         float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (p.h0) v4 = *reinterpret_cast<const float4*>(p.h0 + base + q);
+        if (p.h0 && seg == 0) v4 = *reinterpret_cast<const float4*>(p.h0 + base + q);   // later segments: zero start
         h[q] = v4.x; h[q + 1] = v4.y; h[q + 2] = v4.z; h[q + 3] = v4.w;
+      }
+      if (trans) {                                       // identity columns slice * NV + cg0 .. of the transition
+#pragma unroll
+        for (int q = 0; q < NVT; ++q) h[q] = row == slice * NV + cg0 + q ? 1.f : 0.f;
       }
     }
 #pragma unroll
@@ -314,7 +340,12 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
       const float dec = sc[i];
       const float gam = sc[64 + row];
       float pre[32];
-      load_img32(stage + (row < 64 ? Cfg::OFF_U : Cfg::OFF_O), i, cg0, pre);
+      if (!trans) {
+        load_img32(stage + (row < 64 ? Cfg::OFF_U : Cfg::OFF_O), i, cg0, pre);
+      } else {
+#pragma unroll
+        for (int q = 0; q < 32; ++q) pre[q] = 0.f;
+      }
 
       mbar_wait(bar_mma1, ph, abort_flag, p.spin_limit);
       HA_PROF(chain, 8 * c + 2);
@@ -324,7 +355,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
         for (int c0 = 0; c0 < NVT; c0 += 32) {
           float d[32];
           ld32f(TM1 + lane_base + cg0 + c0, d);
-          if (c0 > 0) load_img32(stage + Cfg::OFF_U, i, cg0 + c0, pre);
+          if (c0 > 0 && !trans) load_img32(stage + Cfg::OFF_U, i, cg0 + c0, pre);
 #pragma unroll
           for (int q = 0; q < 32; ++q) d[q] = (pre[q] - d[q]) * dec;
           if (c0 == 0) HA_PROF(chain, 8 * c + 6);
@@ -340,15 +371,15 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
         // holds one token row, so direct stores would touch 32 lines per instruction); the ragged last chunk
         // of a sequence is stored row by row, since a tile store could not stop at the sequence's end.
         // (32-channel slices keep the direct stores: four per thread, cheaper than the staging's two barriers.)
-        const bool tile_out = NV > 32 && L == kChunk;
-        __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) +
+        const bool tile_out = NV > 32 && L == kChunk && !trans;   // (the tensor map is o's: transition rows go out directly)
+        __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(trans ? p.r_out : p.o) +
                               ((size_t)(tok0 + c * kChunk + i) * p.HV + j) * 128 + (size_t)slice * NV + cg0;
         if (tile_out) named_sync(BAR_O_FREE, NCOMP / 2);
 #pragma unroll
         for (int c0 = 0; c0 < NVT; c0 += 32) {
           float d[32];
           ld32f(TM1 + lane_base + cg0 + c0, d);
-          if (c0 > 0) load_img32(stage + Cfg::OFF_O, i, cg0 + c0, pre);
+          if (c0 > 0 && !trans) load_img32(stage + Cfg::OFF_O, i, cg0 + c0, pre);
 #pragma unroll
           for (int q = 0; q < 32; ++q) d[q] = p.scale * (pre[q] + d[q]);
           if (tile_out) {
@@ -398,11 +429,14 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
       if (blockIdx.x == 0 && tid == 0 && (c == 0 || c == nchunks - 1)) HA_PROF_GT(chain, 700 + c);
     }
 
-    if (p.hT) {
-      const size_t base = (((size_t)n * p.HV + j) * 128 + row) * 128 + (size_t)slice * NV + cg0;
+    // where the end state goes: hT, or with segments the segment's offset b_s / transition Phi_s
+    float* hdst = p.hT ? p.hT + ((size_t)n * p.HV + j) * 128 * 128 : nullptr;
+    if (p.nseg > 1) hdst = (trans ? p.seg_phi : p.seg_b) + (((size_t)n * p.HV + j) * p.nseg + seg) * 128 * 128;
+    if (hdst) {
+      const size_t base = (size_t)row * 128 + (size_t)slice * NV + cg0;
 #pragma unroll
       for (int q = 0; q < NVT; q += 4)
-        *reinterpret_cast<float4*>(p.hT + base + q) = make_float4(h[q], h[q + 1], h[q + 2], h[q + 3]);
+        *reinterpret_cast<float4*>(hdst + base + q) = make_float4(h[q], h[q + 1], h[q + 2], h[q + 3]);
     }
   }
 
@@ -802,7 +836,7 @@ cudaError_t run_variant(const ChainParams* cp, const CUtensorMap* mk, const CUte
 
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                             const CUtensorMap& mk, const CUtensorMap& mo, int nv, int64_t epoch, bool dependent,
-                            uint32_t spin_limit, cudaStream_t stream) {
+                            uint32_t spin_limit, const SegBuffers& sg, cudaStream_t stream) {
   ChainParams cp;
   cp.h0 = a.h0; cp.hT = a.hT; cp.o = a.o;
   cp.seq_tok0 = plan.seq_tok0; cp.seq_len = plan.seq_len; cp.seq_chunk0 = plan.seq_chunk0;
@@ -811,7 +845,8 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   cp.ws = ws; cp.HK = p.HK; cp.HV = p.HV; cp.scale = p.scale; cp.status = a.status_word;
   cp.epoch = epoch;
   cp.spin_limit = spin_limit;
-  const int grid = p.N * p.HV * (128 / nv);
+  cp.nseg = sg.nseg; cp.seg_b = sg.seg_b; cp.seg_phi = sg.seg_phi; cp.r_out = sg.r;
+  const int grid = p.N * p.HV * (128 / nv) * (2 * sg.nseg - 1);
   if (grid == 0) return cudaSuccess;
   return p.variant == HA_LA_KDA ? run_variant<true>(&cp, &mk, &mo, nv, grid, dependent, stream)
                                 : run_variant<false>(&cp, &mk, &mo, nv, grid, dependent, stream);

@@ -49,4 +49,32 @@ inline __host__ TcWorkspace tc_ws_view(void* base, size_t ncj, bool kda) {
   return w;
 }
 
+// Scratch of the segment-parallel state passing, behind the images: per (sequence, V-head) and segment the
+// offset b_s and the transition Phi_s (fp32 128 x 128 each) and the segment's true start state as bf16; per
+// token-head the transition output rows R (bf16 [T][HV][128]).
+struct SegBuffers {
+  int nseg;             // 1: segments are off and the pointers are null
+  float* seg_b;
+  float* seg_phi;
+  __nv_bfloat16* hs;    // [N*HV][nseg][128][128]: start state of segment s (s >= 1)
+  __nv_bfloat16* r;     // [T][HV][128]
+};
+
+inline __host__ size_t tc_seg_bytes(size_t nj, int nseg, size_t rows, int HV) {
+  if (nseg <= 1) return 0;
+  return nj * nseg * 128 * 128 * (4 + 4 + 2) + align_up(rows * HV * 128 * 2, 1024);
+}
+
+inline __host__ SegBuffers tc_seg_view(void* base, size_t nj, int nseg, size_t rows, int HV) {
+  SegBuffers g{nseg, nullptr, nullptr, nullptr, nullptr};
+  if (nseg <= 1) return g;
+  uint8_t* b = reinterpret_cast<uint8_t*>(base);
+  g.seg_b = reinterpret_cast<float*>(b);               b += nj * nseg * 128 * 128 * 4;
+  g.seg_phi = reinterpret_cast<float*>(b);             b += nj * nseg * 128 * 128 * 4;
+  g.hs = reinterpret_cast<__nv_bfloat16*>(b);          b += nj * nseg * 128 * 128 * 2;
+  g.r = reinterpret_cast<__nv_bfloat16*>(b);
+  (void)rows; (void)HV;
+  return g;
+}
+
 }  // namespace ha_la

@@ -179,6 +179,42 @@ def test_bad_cu_seqlens_reports_device_check():
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("variant", ["gdn", "kda"])
+@pytest.mark.parametrize("nseg,nv", [(2, 32), (4, 32), (2, 64), (8, 64)])
+def test_segment_parallel_state_passing(variant, nseg, nv, monkeypatch):
+    """A sequence's chunks cut into segments that are walked at the same time (later segments from a zero state and
+    from the identity, then one affine fix-up per segment).  Slow decay and no decay at all keep the start state of
+    every segment in play -- a wrong start state shows there -- with an initial state, a ragged tail, segment
+    boundaries that do not divide the chunk count, and batched rows."""
+    import paper_2609_32114_b200 as ha
+
+    monkeypatch.setenv("HA_LA_TC_SEGMENTS", str(nseg))
+    monkeypatch.setenv("HA_LA_TC_NV", str(nv))
+    base = W["gdn_layer_4k"] if variant == "gdn" else W["kda_8k"]
+    for lens, shift in (([1100], -4.0), ([700, 700], None), ([130], 2.0)):
+        w = synth.shrink(base, seq_lens=lens, hk=1, hv=2, gate_shift=shift or 0.0, h0_std=0.05)
+        inp = synth.make_inputs(w, seed=91 + nseg)
+        if shift is None:
+            inp["g"][:] = 0
+        a = ha.make_args(variant=variant, dtype="bf16", batch=len(lens), seqlen=lens[0], hk=1, hv=2, dk=128, dv=128)
+        want = nseg if nseg <= (lens[0] + 63) // 64 else None
+        if want:
+            assert ha.ha_la_prefill_num_segments(a) == nseg
+        helpers.check_parity(inp)
+
+
+def test_segments_chosen_only_where_every_run_gets_an_sm():
+    """Host side of the planner: the headline layer (16 heads) keeps one segment, a long sequence with two heads
+    is cut up, packed batches never are."""
+    import paper_2609_32114_b200 as ha
+
+    mk = lambda **kw: ha.make_args(**dict(dict(variant="gdn", dtype="bf16", batch=1, seqlen=4096, hk=16, hv=16,
+                                               dk=128, dv=128), **kw))
+    assert ha.ha_la_prefill_num_segments(mk()) == 1
+    assert ha.ha_la_prefill_num_segments(mk(seqlen=16384, hk=2, hv=2)) > 1
+    assert ha.ha_la_prefill_num_segments(mk(seqlen=16384, hk=2, hv=2, num_seqs=2)) == 1
+
+
 def test_bounded_wait_runs_out_and_reports_timeout():
     """Every device-side wait is bounded.  The test hook launches the sequential kernel alone, waiting per chunk for
     flags that nothing publishes, with a limit of a few thousand polls: the wait must run out, the status word must
