@@ -1,6 +1,11 @@
 """Builds libha_la.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
-    python -m paper_2609_32114_b200.build [--force] [--verbose]
+    python -m paper_2609_32114_b200.build [--force] [--verbose] [--profile]
+
+--profile builds a second library, libha_la_prof.so, with -DHA_LA_PROFILE_PHASES: the tensor-core kernels then
+record clock64 / %globaltimer stamps at their phase boundaries (csrc/prof.cuh) and the library exports
+ha_la_debug_read_prof_prep / _chain to read them; `python -m paper_2609_32114_b200.prof_phases` prints them.
+The normal library contains none of this (the macros expand to nothing).
 
 Objects are cached under paper_2609_32114_b200/build/ and rebuilt when their source, any
 header, or this script changes; translation units compile in parallel.
@@ -77,5 +82,17 @@ def build(force: bool = False, verbose: bool = False, extra_flags=(), lib_path: 
     return lib_path
 
 
+PROF_LIB = os.path.join(PKG, "libha_la_prof.so")
+
+
+def build_profile(force: bool = False, verbose: bool = False) -> str:
+    """The instrumented developer build (see the module docstring)."""
+    return build(force=force, verbose=verbose, extra_flags=["-DHA_LA_PROFILE_PHASES"], lib_path=PROF_LIB,
+                 obj_dir=os.path.join(PKG, "build_prof"))
+
+
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    if "--profile" in sys.argv:
+        print(build_profile(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    else:
+        print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))

@@ -1,5 +1,6 @@
-// Optional phase timestamps for kernel tuning.  Compiled in only with -DHA_LA_PROFILE_PHASES (a
-// developer build); in the normal build both macros expand to nothing.
+// Optional phase timestamps for kernel tuning.  Compiled in only with -DHA_LA_PROFILE_PHASES (the developer build
+// `python -m paper_2609_32114_b200.build --profile`, read back by `python -m paper_2609_32114_b200.prof_phases`);
+// in the normal build every macro expands to nothing.
 #pragma once
 #ifdef HA_LA_PROFILE_PHASES
 #define HA_PROF_DECL(name)                                                                        \

@@ -172,8 +172,9 @@ TcPlan plan_tc(const Problem& p) {
   // Segment-parallel state passing (equal-length rows, sliced kernels, back to back with the prep kernel): a
   // sequence's chain is cut into nseg segments that run at once; a later segment costs three times the columns of
   // the first (its own from a zero state plus 128 transition columns), so it only pays while all those CTAs have an
-  // SM each, i.e. for few heads and long sequences.  Costs measured on B200: the chain's per-chunk times above, some
-  // 3 us per segment for the start states and about a quarter of a microsecond of one SM per corrected chunk-head.
+  // SM each, i.e. for few heads and long sequences.  Costs measured on B200: the chain's per-chunk times above,
+  // 7 us + 5.5 us per further segment for the start states (S - 1 products of 128^3 in turn) and 9 us + 25 ns per
+  // corrected chunk-head for the outputs.
   int forced_seg = 0;
   if (const char* e = getenv("HA_LA_TC_SEGMENTS")) {
     const int v = atoi(e);
@@ -190,7 +191,7 @@ TcPlan plan_tc(const Problem& p) {
         const double cpseg = (double)(long long)((longest + nseg - 1) / nseg);
         const double waves = (double)((ctas + sms - 1) / sms);
         const double later = items * (1.0 - 1.0 / nseg);
-        const double t = prep_us + waves * cpseg * per_chunk_us[w] + 4.0 + 3.0 * (nseg - 1) + 5.0 + later * 0.25 / sms;
+        const double t = prep_us + waves * cpseg * per_chunk_us[w] + (7.0 + 5.5 * (nseg - 1)) + (9.0 + 0.025 * later);
         if (t < best || (forced_seg && plan.nseg != forced_seg)) { best = t; plan = TcPlan{widths[w], false, nseg}; }
       }
     }

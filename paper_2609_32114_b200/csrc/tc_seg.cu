@@ -26,108 +26,140 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-constexpr int kFixCols = 16;             // state columns per CTA of the fix-up kernel
-constexpr int kPhiLd = 129;              // padded row stride (floats) of the transition in shared memory
-constexpr size_t kFixSmem = (size_t)128 * kPhiLd * 4 + 128 * kFixCols * 4;
+// h_{s+1} = Phi_s h_s + b_s, s = 1 .. S-1 in turn, for 32 of the 128 state columns per CTA (columns are
+// independent).  Eight warps, 16 state rows each; the product runs on the legacy tensor path in TF32 (wmma
+// m16n16k8, fp32 accumulation starting from b_s): Phi_s and h_s round to 11 significant bits, finer than the bf16
+// operands of every other product of the path.  The transition of a segment (64 KiB) goes through shared memory:
+// coalesced 16-byte loads, all of a thread's in flight together, the next segment's fetched under this one's product.
+constexpr int kFixCols = 32;             // state columns per CTA
+constexpr int kPhiLd = 128 + 4;          // row strides (floats) in shared memory
+constexpr int kHLd = kFixCols + 4;
+constexpr size_t kFixSmem = (size_t)128 * kPhiLd * 4 + (size_t)128 * kHLd * 4;
 
 __global__ void __launch_bounds__(256) seg_fix_kernel(SegBuffers sg, float* hT) {
-  extern __shared__ __align__(16) float fsm[];
-  float* sPhi = fsm;                     // [128][kPhiLd]: Phi_s, whole (every thread walks one row of it)
-  float* sh = fsm + 128 * kPhiLd;        // [128][kFixCols]: h_s, this CTA's columns
+  using namespace nvcuda;
+  extern __shared__ __align__(32) float fsm[];
+  float* sPhi = fsm;                     // [128][kPhiLd]: Phi_s
+  float* sh = fsm + 128 * kPhiLd;        // [128][kHLd]: h_s, this CTA's columns
   const int nj = blockIdx.x;
   const int x0 = blockIdx.y * kFixCols;
-  const int i = threadIdx.x & 127;       // state row
-  const int xh = (threadIdx.x >> 7) * 8; // which 8 of the 16 columns
+  const int tid = threadIdx.x, warp = tid >> 5;
   const size_t seg_stride = 128 * 128;
   const float* b = sg.seg_b + (size_t)nj * sg.nseg * seg_stride;
   const float* phi = sg.seg_phi + (size_t)nj * sg.nseg * seg_stride;
   __nv_bfloat16* hs = sg.hs + (size_t)nj * sg.nseg * seg_stride;
-  float h[8];
+  const int hr = tid >> 1, hc = (tid & 1) * 16;          // this thread's 16 values of the 128 x 32 tile (copies)
+  asm volatile("griddepcontrol.wait;" ::: "memory");     // (launched as a programmatic dependent of the chain kernel)
+  float4 t[16];
   {
-    const float4 a0 = *reinterpret_cast<const float4*>(b + (size_t)i * 128 + x0 + xh);
-    const float4 a1 = *reinterpret_cast<const float4*>(b + (size_t)i * 128 + x0 + xh + 4);
-    h[0] = a0.x; h[1] = a0.y; h[2] = a0.z; h[3] = a0.w; h[4] = a1.x; h[5] = a1.y; h[6] = a1.z; h[7] = a1.w;   // h_1
-  }
-  for (int s = 1; s < sg.nseg; ++s) {
-    // the whole transition of this segment: coalesced 16-byte loads, all in flight together
-    const float4* g4 = reinterpret_cast<const float4*>(phi + (size_t)s * seg_stride);
-    float4 t[16];
+    const float4* g4 = reinterpret_cast<const float4*>(phi + seg_stride);
 #pragma unroll
-    for (int q = 0; q < 16; ++q) t[q] = g4[q * 256 + threadIdx.x];
-    float acc[8];
-    {
-      const float* bs = b + (size_t)s * seg_stride + (size_t)i * 128 + x0 + xh;
-      const float4 a0 = *reinterpret_cast<const float4*>(bs), a1 = *reinterpret_cast<const float4*>(bs + 4);
-      acc[0] = a0.x; acc[1] = a0.y; acc[2] = a0.z; acc[3] = a0.w; acc[4] = a1.x; acc[5] = a1.y; acc[6] = a1.z; acc[7] = a1.w;
-    }
+    for (int q = 0; q < 16; ++q) t[q] = g4[q * 256 + tid];
+  }
+  // h_1 = end state of segment 0 (which started from the real initial state)
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    *reinterpret_cast<float4*>(sh + hr * kHLd + hc + 4 * q) = *reinterpret_cast<const float4*>(b + (size_t)hr * 128 + x0 + hc + 4 * q);
+  for (int s = 1; s < sg.nseg; ++s) {
 #pragma unroll
     for (int q = 0; q < 16; ++q) {
-      const int e = (q * 256 + threadIdx.x) * 4, r = e >> 7, c = e & 127;
-      float* d = sPhi + r * kPhiLd + c;
-      d[0] = t[q].x; d[1] = t[q].y; d[2] = t[q].z; d[3] = t[q].w;
+      const int e = (q * 256 + tid) * 4;
+      *reinterpret_cast<float4*>(sPhi + (e >> 7) * kPhiLd + (e & 127)) = t[q];
     }
-    const uint4 w = make_uint4(pack2(h[0], h[1]), pack2(h[2], h[3]), pack2(h[4], h[5]), pack2(h[6], h[7]));
-    *reinterpret_cast<uint4*>(hs + (size_t)s * seg_stride + (size_t)i * 128 + x0 + xh) = w;   // h_s for the output kernel
+    __syncthreads();                                     // Phi_s and h_s are in shared memory
+    if (s + 1 < sg.nseg) {
+      const float4* g4 = reinterpret_cast<const float4*>(phi + (size_t)(s + 1) * seg_stride);
 #pragma unroll
-    for (int q = 0; q < 8; ++q) sh[i * kFixCols + xh + q] = h[q];
-    __syncthreads();
-    const float* prow = sPhi + i * kPhiLd;
-#pragma unroll 8
-    for (int v = 0; v < 128; ++v) {
-      const float f = prow[v];
-      const float4 s0 = *reinterpret_cast<const float4*>(sh + v * kFixCols + xh);
-      const float4 s1 = *reinterpret_cast<const float4*>(sh + v * kFixCols + xh + 4);
-      acc[0] = fmaf(f, s0.x, acc[0]); acc[1] = fmaf(f, s0.y, acc[1]); acc[2] = fmaf(f, s0.z, acc[2]); acc[3] = fmaf(f, s0.w, acc[3]);
-      acc[4] = fmaf(f, s1.x, acc[4]); acc[5] = fmaf(f, s1.y, acc[5]); acc[6] = fmaf(f, s1.z, acc[6]); acc[7] = fmaf(f, s1.w, acc[7]);
+      for (int q = 0; q < 16; ++q) t[q] = g4[q * 256 + tid];
     }
-    __syncthreads();
+    {                                                    // h_s as bf16, for the output kernel
+      uint32_t w[8];
 #pragma unroll
-    for (int q = 0; q < 8; ++q) h[q] = acc[q];
+      for (int q = 0; q < 8; ++q) w[q] = pack2(sh[hr * kHLd + hc + 2 * q], sh[hr * kHLd + hc + 2 * q + 1]);
+      uint4* d = reinterpret_cast<uint4*>(hs + (size_t)s * seg_stride + (size_t)hr * 128 + x0 + hc);
+      d[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      d[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+    wmma::fragment<wmma::accumulator, 16, 16, 8, float> acc[2];
+#pragma unroll
+    for (int x = 0; x < 2; ++x)
+      wmma::load_matrix_sync(acc[x], b + (size_t)s * seg_stride + (size_t)(warp * 16) * 128 + x0 + x * 16, 128, wmma::mem_row_major);
+#pragma unroll 4
+    for (int k = 0; k < 16; ++k) {
+      wmma::fragment<wmma::matrix_a, 16, 16, 8, wmma::precision::tf32, wmma::row_major> fa;
+      wmma::load_matrix_sync(fa, sPhi + (warp * 16) * kPhiLd + k * 8, kPhiLd);
+#pragma unroll
+      for (int e = 0; e < fa.num_elements; ++e) fa.x[e] = wmma::__float_to_tf32(fa.x[e]);
+#pragma unroll
+      for (int x = 0; x < 2; ++x) {
+        wmma::fragment<wmma::matrix_b, 16, 16, 8, wmma::precision::tf32, wmma::row_major> fb;
+        wmma::load_matrix_sync(fb, sh + (k * 8) * kHLd + x * 16, kHLd);
+#pragma unroll
+        for (int e = 0; e < fb.num_elements; ++e) fb.x[e] = wmma::__float_to_tf32(fb.x[e]);
+        wmma::mma_sync(acc[x], fa, fb, acc[x]);
+      }
+    }
+    __syncthreads();                                     // every warp has read h_s and Phi_s
+#pragma unroll
+    for (int x = 0; x < 2; ++x) wmma::store_matrix_sync(sh + (warp * 16) * kHLd + x * 16, acc[x], kHLd, wmma::mem_row_major);
+    __syncthreads();                                     // h_{s+1} is complete
   }
   if (hT) {
-    float* d = hT + (size_t)nj * seg_stride + (size_t)i * 128 + x0 + xh;
-    *reinterpret_cast<float4*>(d) = make_float4(h[0], h[1], h[2], h[3]);
-    *reinterpret_cast<float4*>(d + 4) = make_float4(h[4], h[5], h[6], h[7]);
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      *reinterpret_cast<float4*>(hT + (size_t)nj * seg_stride + (size_t)hr * 128 + x0 + hc + 4 * q) =
+          *reinterpret_cast<const float4*>(sh + hr * kHLd + hc + 4 * q);
   }
 }
 
-// o[t][:] += R[t][:] h_s  for the 64 tokens of one chunk of one V-head.  Four warps, 16 token rows each; R, h_s and
-// the result go through shared memory (operand loads straight from global memory were latency-bound: 64 small tile
-// loads per warp).
+// o[t][:] += R[t][:] h_s  for two neighbouring chunks (128 tokens) of one later segment of one V-head.  Eight warps,
+// 16 token rows each; h_s (loaded once for both chunks), R and the result go through shared memory (operand loads
+// straight from global memory were latency-bound: 64 small tile loads per warp).
 constexpr int kLdR = 128 + 8, kLdC = 64 + 4;
-constexpr size_t kOutSmem = (size_t)(64 + 128) * kLdR * 2 + (size_t)4 * 16 * kLdC * 4;
+constexpr size_t kOutSmem = (size_t)(128 + 128) * kLdR * 2 + (size_t)8 * 16 * kLdC * 4;
 
-__global__ void __launch_bounds__(128) seg_out_kernel(SegBuffers sg, __nv_bfloat16* o, int T_row, int cps, int HV) {
+__global__ void __launch_bounds__(256) seg_out_kernel(SegBuffers sg, __nv_bfloat16* o, int T_row, int HV) {
   using namespace nvcuda;
   extern __shared__ __align__(32) uint8_t osm[];
-  __nv_bfloat16* sR = reinterpret_cast<__nv_bfloat16*>(osm);                  // [64][kLdR]
-  __nv_bfloat16* sB = sR + 64 * kLdR;                                          // [128][kLdR]: h_s
-  float* sC = reinterpret_cast<float*>(sB + 128 * kLdR);                       // [4][16][kLdC]
-  const int slot = blockIdx.x;                           // chunk slot: chunk cc of batch row n
-  const int j = blockIdx.y;
-  const int n = slot / cps, cc = slot % cps;
+  __nv_bfloat16* sR = reinterpret_cast<__nv_bfloat16*>(osm);                  // [128][kLdR]: two chunks of R
+  __nv_bfloat16* sB = sR + 128 * kLdR;                                         // [128][kLdR]: h_s
+  float* sC = reinterpret_cast<float*>(sB + 128 * kLdR);                       // [8][16][kLdC]
   const int nch = (T_row + kChunk - 1) / kChunk;
   const int cpseg = (nch + sg.nseg - 1) / sg.nseg;
-  const int seg = cc / cpseg;
-  if (cc >= nch || seg == 0) return;                     // segment 0 ran from the real start state
-  const int L = min(kChunk, T_row - cc * kChunk);
-  const size_t row0 = (size_t)n * T_row + (size_t)cc * kChunk;
+  const int pairs = (cpseg + 1) / 2;                     // chunk pairs per segment
+  const int j = blockIdx.y;
+  const int pair = blockIdx.x % pairs;
+  const int seg = 1 + (blockIdx.x / pairs) % (sg.nseg - 1);
+  const int n = blockIdx.x / (pairs * (sg.nseg - 1));
+  const int cc0 = seg * cpseg + 2 * pair;                // first chunk of the pair
+  const int cend = min((seg + 1) * cpseg, nch);          // end of the segment
+  asm volatile("griddepcontrol.wait;" ::: "memory");     // (programmatic dependent of the fix-up kernel)
+  if (cc0 >= cend) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const size_t row0 = (size_t)n * T_row + (size_t)cc0 * kChunk;
+  const int rows_here = min(min(cend - cc0, 2) * kChunk, T_row - cc0 * kChunk);   // valid token rows of the pair
   const __nv_bfloat16* hs = sg.hs + (((size_t)n * HV + j) * sg.nseg + seg) * 128 * 128;
-  // R tile (rows past the end of the sequence as zeros) and h_s -> shared memory
-#pragma unroll 4
-  for (int idx = tid; idx < 64 * 16; idx += 128) {
-    const int t = idx >> 4, p8 = idx & 15;
-    uint4 w = make_uint4(0u, 0u, 0u, 0u);
-    if (t < L) w = *reinterpret_cast<const uint4*>(sg.r + ((row0 + t) * HV + j) * 128 + p8 * 8);
-    *reinterpret_cast<uint4*>(sR + t * kLdR + p8 * 8) = w;
-  }
-#pragma unroll 4
-  for (int idx = tid; idx < 128 * 16; idx += 128) {
-    const int v = idx >> 4, p8 = idx & 15;
-    *reinterpret_cast<uint4*>(sB + v * kLdR + p8 * 8) = *reinterpret_cast<const uint4*>(hs + (size_t)v * 128 + p8 * 8);
+  {
+    uint4 w[8], r[8];                                    // all loads of a thread in flight together
+#pragma unroll
+    for (int q = 0; q < 8; ++q) w[q] = *reinterpret_cast<const uint4*>(hs + (size_t)(q * 256 + tid) * 8);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int idx = q * 256 + tid, t = idx >> 4, p8 = idx & 15;
+      r[q] = make_uint4(0u, 0u, 0u, 0u);                 // rows past the pair's end as zeros
+      if (t < rows_here) r[q] = *reinterpret_cast<const uint4*>(sg.r + ((row0 + t) * HV + j) * 128 + p8 * 8);
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int idx = q * 256 + tid;
+      *reinterpret_cast<uint4*>(sB + (idx >> 4) * kLdR + (idx & 15) * 8) = w[q];
+      *reinterpret_cast<uint4*>(sR + (idx >> 4) * kLdR + (idx & 15) * 8) = r[q];
+    }
   }
   __syncthreads();
+  const int rows = min(16, rows_here - warp * 16);       // this warp's valid rows
+  if (rows <= 0) return;
   wmma::fragment<wmma::accumulator, 16, 16, 16, float> acc[8];
 #pragma unroll
   for (int x = 0; x < 8; ++x) wmma::fill_fragment(acc[x], 0.f);
@@ -151,7 +183,6 @@ __global__ void __launch_bounds__(128) seg_out_kernel(SegBuffers sg, __nv_bfloat
     // after the other, a memory latency each)
     __nv_bfloat162* op = reinterpret_cast<__nv_bfloat162*>(o + ((row0 + warp * 16) * HV + j) * 128 + half * 64 + lane * 2);
     const size_t rstride = (size_t)HV * 64;              // one token row further, in bf16 pairs
-    const int rows = min(16, L - warp * 16);
     __nv_bfloat162 ov[16];
 #pragma unroll
     for (int r = 0; r < 16; ++r)
@@ -177,15 +208,29 @@ cudaError_t launch_tc_seg_fix(const Problem& p, const ha_la_prefill_args& a, con
   cudaError_t ce = cudaFuncSetAttribute(seg_fix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFixSmem);
   if (ce == cudaSuccess) ce = cudaFuncSetAttribute(seg_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kOutSmem);
   if (ce != cudaSuccess) return ce;
+  // Both kernels are launched as programmatic dependents of the kernel before them (each waits for it on the
+  // device before its first read), which hides their launch latency under that kernel's tail.
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = g_timer ? 0 : 1;                        // (per-kernel timing wants one kernel at a time)
   timer_mark(stream, "tc_seg_fix");
-  seg_fix_kernel<<<dim3((unsigned)(p.N * p.HV), 128 / kFixCols), 256, kFixSmem, stream>>>(sg, a.hT);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  cfg.gridDim = dim3((unsigned)(p.N * p.HV), 128 / kFixCols);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = kFixSmem;
+  ce = cudaLaunchKernelEx(&cfg, seg_fix_kernel, sg, a.hT);
+  if (ce != cudaSuccess) return ce;
+  const int nch = (p.T_row + kChunk - 1) / kChunk;
+  const int cpseg = (nch + sg.nseg - 1) / sg.nseg;
+  if (nch <= cpseg) return cudaSuccess;                  // (everything is in segment 0)
   timer_mark(stream, "tc_seg_out");
-  const int cps = p.max_seq_chunks > 0 ? p.max_seq_chunks : 1;
-  seg_out_kernel<<<dim3((unsigned)(p.N * cps), (unsigned)p.HV), 128, kOutSmem, stream>>>(
-      sg, reinterpret_cast<__nv_bfloat16*>(a.o), p.T_row, cps, p.HV);
-  return cudaGetLastError();
+  cfg.gridDim = dim3((unsigned)(p.N * (sg.nseg - 1) * ((cpseg + 1) / 2)), (unsigned)p.HV);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = kOutSmem;
+  return cudaLaunchKernelEx(&cfg, seg_out_kernel, sg, reinterpret_cast<__nv_bfloat16*>(a.o), p.T_row, p.HV);
 }
 
 }  // namespace ha_la
