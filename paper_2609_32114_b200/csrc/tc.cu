@@ -26,7 +26,8 @@ cudaError_t launch_tc_prep(const Problem& p, const ha_la_prefill_args& a, PlanVi
 cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const TcWorkspace& ws,
                             const CUtensorMap& mk, const CUtensorMap& mo, int nv, int64_t epoch, bool dependent,
                             uint32_t spin_limit, const SegBuffers& sg, cudaStream_t stream);
-cudaError_t launch_tc_seg_fix(const Problem& p, const ha_la_prefill_args& a, const SegBuffers& sg, cudaStream_t stream);
+cudaError_t launch_tc_seg_fix(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const SegBuffers& sg,
+                              cudaStream_t stream);
 
 cudaError_t configure_tc_prep(const Problem& p);
 cudaError_t configure_tc_chain(const Problem& p, int nv);
@@ -180,7 +181,7 @@ TcPlan plan_tc(const Problem& p) {
     const int v = atoi(e);
     if (v == 1 || v == 2 || v == 4 || v == 8) forced_seg = v;
   }
-  if (!p.varlen && forced_seg != 1 && longest >= 2) {
+  if ((!p.varlen || forced_seg > 1) && forced_seg != 1 && longest >= 2) {
     for (int w = 0; w < 2; ++w) {                          // 32- and 64-channel slices
       if (forced_nv && widths[w] != forced_nv) continue;
       for (int nseg = 2; nseg <= 8; nseg *= 2) {
@@ -209,7 +210,7 @@ bool tc_supported(const Problem& p) {
 // that was sized before they were set)
 size_t tc_workspace_bytes(const Problem& p) {
   const size_t img = tc_ws_bytes_for((size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
-  return img + (p.varlen ? 0 : tc_seg_bytes((size_t)p.N * p.HV, 8, (size_t)p.T_total, p.HV));
+  return img + tc_seg_bytes((size_t)p.N * p.HV, 8, (size_t)p.T_total, p.HV);
 }
 
 int tc_num_launches(const Problem& p) { return plan_tc(p).nseg > 1 ? 4 : 2; }
@@ -258,7 +259,7 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
   if (e != cudaSuccess) return e;
   e = launch_tc_chain(p, a, plan, ws, mk, mo, nv, epoch, /*dependent=*/g_timer == nullptr, kDefaultSpinLimit, sg, stream);
   if (e != cudaSuccess) return e;
-  return launch_tc_seg_fix(p, a, sg, stream);
+  return launch_tc_seg_fix(p, a, plan, sg, stream);
 }
 
 // Test hook behind ha_la_debug_wait_timeout: the sequential kernel alone, in the concurrent mode, with an epoch that

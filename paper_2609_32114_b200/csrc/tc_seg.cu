@@ -36,7 +36,7 @@ constexpr int kPhiLd = 128 + 4;          // row strides (floats) in shared memor
 constexpr int kHLd = kFixCols + 4;
 constexpr size_t kFixSmem = (size_t)128 * kPhiLd * 4 + (size_t)128 * kHLd * 4;
 
-__global__ void __launch_bounds__(256) seg_fix_kernel(SegBuffers sg, float* hT) {
+__global__ void __launch_bounds__(256) seg_fix_kernel(SegBuffers sg, float* hT, int T_row, int HV, const int32_t* seq_len) {
   using namespace nvcuda;
   extern __shared__ __align__(32) float fsm[];
   float* sPhi = fsm;                     // [128][kPhiLd]: Phi_s
@@ -49,6 +49,11 @@ __global__ void __launch_bounds__(256) seg_fix_kernel(SegBuffers sg, float* hT) 
   const float* phi = sg.seg_phi + (size_t)nj * sg.nseg * seg_stride;
   __nv_bfloat16* hs = sg.hs + (size_t)nj * sg.nseg * seg_stride;
   const int hr = tid >> 1, hc = (tid & 1) * 16;          // this thread's 16 values of the 128 x 32 tile (copies)
+  // segments past the end of a short sequence are empty: their transition is the identity and the state passes
+  // through untouched (bit for bit, which the TF32 product would not do)
+  const int len = seq_len ? seq_len[nj / HV] : T_row;
+  const int nch = (len + kChunk - 1) / kChunk;
+  const int cpseg = (nch + sg.nseg - 1) / sg.nseg;
   asm volatile("griddepcontrol.wait;" ::: "memory");     // (launched as a programmatic dependent of the chain kernel)
   float4 t[16];
   {
@@ -80,6 +85,7 @@ __global__ void __launch_bounds__(256) seg_fix_kernel(SegBuffers sg, float* hT) 
       d[0] = make_uint4(w[0], w[1], w[2], w[3]);
       d[1] = make_uint4(w[4], w[5], w[6], w[7]);
     }
+    if (s * cpseg >= nch) continue;                      // empty segment (the same for every thread of the CTA)
     wmma::fragment<wmma::accumulator, 16, 16, 8, float> acc[2];
 #pragma unroll
     for (int x = 0; x < 2; ++x)
@@ -119,26 +125,29 @@ __global__ void __launch_bounds__(256) seg_fix_kernel(SegBuffers sg, float* hT) 
 constexpr int kLdR = 128 + 8, kLdC = 64 + 4;
 constexpr size_t kOutSmem = (size_t)(128 + 128) * kLdR * 2 + (size_t)8 * 16 * kLdC * 4;
 
-__global__ void __launch_bounds__(256) seg_out_kernel(SegBuffers sg, __nv_bfloat16* o, int T_row, int HV) {
+__global__ void __launch_bounds__(256) seg_out_kernel(SegBuffers sg, __nv_bfloat16* o, int T_row, int HV, int pairs,
+                                                      const int32_t* seq_tok0, const int32_t* seq_len) {
   using namespace nvcuda;
   extern __shared__ __align__(32) uint8_t osm[];
   __nv_bfloat16* sR = reinterpret_cast<__nv_bfloat16*>(osm);                  // [128][kLdR]: two chunks of R
   __nv_bfloat16* sB = sR + 128 * kLdR;                                         // [128][kLdR]: h_s
   float* sC = reinterpret_cast<float*>(sB + 128 * kLdR);                       // [8][16][kLdC]
-  const int nch = (T_row + kChunk - 1) / kChunk;
-  const int cpseg = (nch + sg.nseg - 1) / sg.nseg;
-  const int pairs = (cpseg + 1) / 2;                     // chunk pairs per segment
+  // `pairs` = chunk pairs per segment of the longest sequence the grid was sized for; shorter sequences leave CTAs idle
   const int j = blockIdx.y;
   const int pair = blockIdx.x % pairs;
   const int seg = 1 + (blockIdx.x / pairs) % (sg.nseg - 1);
   const int n = blockIdx.x / (pairs * (sg.nseg - 1));
+  const int len = seq_len ? seq_len[n] : T_row;          // (packed batches: the plan kernel's per-sequence table)
+  const int tok0 = seq_tok0 ? seq_tok0[n] : n * T_row;
+  const int nch = (len + kChunk - 1) / kChunk;
+  const int cpseg = (nch + sg.nseg - 1) / sg.nseg;
   const int cc0 = seg * cpseg + 2 * pair;                // first chunk of the pair
   const int cend = min((seg + 1) * cpseg, nch);          // end of the segment
   asm volatile("griddepcontrol.wait;" ::: "memory");     // (programmatic dependent of the fix-up kernel)
   if (cc0 >= cend) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const size_t row0 = (size_t)n * T_row + (size_t)cc0 * kChunk;
-  const int rows_here = min(min(cend - cc0, 2) * kChunk, T_row - cc0 * kChunk);   // valid token rows of the pair
+  const size_t row0 = (size_t)tok0 + (size_t)cc0 * kChunk;
+  const int rows_here = min(min(cend - cc0, 2) * kChunk, len - cc0 * kChunk);     // valid token rows of the pair
   const __nv_bfloat16* hs = sg.hs + (((size_t)n * HV + j) * sg.nseg + seg) * 128 * 128;
   {
     uint4 w[8], r[8];                                    // all loads of a thread in flight together
@@ -202,7 +211,8 @@ __global__ void __launch_bounds__(256) seg_out_kernel(SegBuffers sg, __nv_bfloat
 }  // namespace
 
 // Both kernels, behind the chain kernel on the same stream.
-cudaError_t launch_tc_seg_fix(const Problem& p, const ha_la_prefill_args& a, const SegBuffers& sg, cudaStream_t stream) {
+cudaError_t launch_tc_seg_fix(const Problem& p, const ha_la_prefill_args& a, PlanView plan, const SegBuffers& sg,
+                              cudaStream_t stream) {
   if (sg.nseg <= 1 || p.N * p.HV == 0) return cudaSuccess;
   // (per device and idempotent; a few microseconds on the host, on a path that is already several launches long)
   cudaError_t ce = cudaFuncSetAttribute(seg_fix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFixSmem);
@@ -221,16 +231,18 @@ cudaError_t launch_tc_seg_fix(const Problem& p, const ha_la_prefill_args& a, con
   cfg.gridDim = dim3((unsigned)(p.N * p.HV), 128 / kFixCols);
   cfg.blockDim = dim3(256);
   cfg.dynamicSmemBytes = kFixSmem;
-  ce = cudaLaunchKernelEx(&cfg, seg_fix_kernel, sg, a.hT);
+  ce = cudaLaunchKernelEx(&cfg, seg_fix_kernel, sg, a.hT, p.T_row, p.HV, (const int32_t*)plan.seq_len);
   if (ce != cudaSuccess) return ce;
-  const int nch = (p.T_row + kChunk - 1) / kChunk;
+  const int nch = p.max_seq_chunks;                      // longest sequence (a bound, for packed batches)
   const int cpseg = (nch + sg.nseg - 1) / sg.nseg;
   if (nch <= cpseg) return cudaSuccess;                  // (everything is in segment 0)
+  const int pairs = (cpseg + 1) / 2;
   timer_mark(stream, "tc_seg_out");
-  cfg.gridDim = dim3((unsigned)(p.N * (sg.nseg - 1) * ((cpseg + 1) / 2)), (unsigned)p.HV);
+  cfg.gridDim = dim3((unsigned)(p.N * (sg.nseg - 1) * pairs), (unsigned)p.HV);
   cfg.blockDim = dim3(256);
   cfg.dynamicSmemBytes = kOutSmem;
-  return cudaLaunchKernelEx(&cfg, seg_out_kernel, sg, reinterpret_cast<__nv_bfloat16*>(a.o), p.T_row, p.HV);
+  return cudaLaunchKernelEx(&cfg, seg_out_kernel, sg, reinterpret_cast<__nv_bfloat16*>(a.o), p.T_row, p.HV, pairs,
+                            (const int32_t*)plan.seq_tok0, (const int32_t*)plan.seq_len);
 }
 
 }  // namespace ha_la

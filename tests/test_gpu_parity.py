@@ -203,6 +203,22 @@ def test_segment_parallel_state_passing(variant, nseg, nv, monkeypatch):
         helpers.check_parity(inp)
 
 
+@pytest.mark.parametrize("variant", ["gdn", "kda"])
+@pytest.mark.parametrize("nseg", [2, 4])
+def test_segments_on_a_packed_batch(variant, nseg, monkeypatch):
+    """Packed batches are never cut into segments by the planner, but the kernels take them (HA_LA_TC_SEGMENTS
+    forces it): every sequence is cut into the same number of segments, so short and empty sequences end up with
+    empty segments, and there are more runs than SMs."""
+    monkeypatch.setenv("HA_LA_TC_SEGMENTS", str(nseg))
+    base = W["gdn_varlen"] if variant == "gdn" else W["kda_8k"]
+    w = synth.shrink(base, seq_lens=[700, 0, 65, 1500, 130, 1], hk=2, hv=4, gate_shift=-3.0, h0_std=0.05, varlen=True)
+    inp = synth.make_inputs(w, seed=97 + nseg)
+    o, hT, status = helpers.run_gpu(inp)
+    assert status == 0
+    np.testing.assert_array_equal(hT[1], inp["h0"][1].astype(np.float64))     # empty sequence: hT = h0 exactly
+    helpers.check_parity(inp)
+
+
 def test_segments_chosen_only_where_every_run_gets_an_sm():
     """Host side of the planner: the headline layer (16 heads) keeps one segment, a long sequence with two heads
     is cut up, packed batches never are."""
