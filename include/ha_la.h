@@ -58,7 +58,7 @@
  * work is launched, never the result): HA_LA_FORCE_SIMT=1 (read once) sends every shape
  * to the fp32 CUDA-core kernel; HA_LA_TC_NV=32|64|128 fixes the slice width of the
  * sequential kernel; HA_LA_TC_OVERLAP=0|2 forbids / forces running the two tensor-core
- * kernels side by side; HA_LA_TC_SEGMENTS=1|2|4 fixes the number of segments a head's
+ * kernels side by side; HA_LA_TC_SEGMENTS=1|2|4|8 fixes the number of segments a head's
  * chunk sequence is split into.  Production callers leave them unset.
  */
 #ifndef HA_LA_H_
@@ -144,7 +144,7 @@ int ha_la_prefill_launch_plan(const ha_la_prefill_args* args, int* slice_width, 
 /* Segments per sequence ha_la_prefill would use for these shapes (host only; 1 = the chunks of a sequence are
  * walked strictly in order; 0 if the shapes are unsupported).  With S > 1 a sequence's chunks are cut into S
  * runs that are walked at the same time -- the Chunk-Seg-Seg mapping the paper describes for its FlashQLA
- * baseline (Section 4.1): later segments start from a zero state and from the identity, and their true start
+ * baseline (Section "Head-Level Mapping with Cross-Operator Fusion"): later segments start from a zero state and from the identity, and their true start
  * states, final state and outputs follow from one affine fix-up per segment.  Chosen only for equal-length rows
  * with so few (sequence, head) pairs that every run still gets an SM; HA_LA_TC_SEGMENTS overrides it.            */
 int ha_la_prefill_num_segments(const ha_la_prefill_args* args);
