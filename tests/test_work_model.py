@@ -23,3 +23,19 @@ def test_algorithmic_work_of_the_headline_workload():
     assert synth.algorithmic_bytes(w, 4096, 1) == 4096 * 16512 + 16 * 128 * 128 * 4   # 68.68 MB
     k = synth.WORKLOADS["kda_8k"]
     assert synth.algorithmic_bytes(k, 8192, 1) == 8192 * 32 * 1540 + 32 * 128 * 128 * 4
+
+
+def test_traffic_table_is_rebuilt_from_the_committed_summaries():
+    """profiles/traffic.json (what bench.py reports as `roofline.traffic`) is exactly what the summary tool derives
+    from the ncu summaries beside it: no hand-copied constants."""
+    import json
+    import os
+
+    from paper_2609_32114_b200 import ncu_summary
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with open(os.path.join(root, "profiles", "traffic.json")) as f:
+        stored = json.load(f)
+    assert stored == json.loads(json.dumps(ncu_summary.traffic()))
+    chain = stored["gdn_layer_4k"]["tc_chain"]
+    assert chain["dram_read"] > 0 and chain["source"].endswith(".md")
