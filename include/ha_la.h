@@ -59,7 +59,9 @@
  * to the fp32 CUDA-core kernel; HA_LA_TC_NV=32|64|128 fixes the slice width of the
  * sequential kernel; HA_LA_TC_OVERLAP=0|2 forbids / forces running the two tensor-core
  * kernels side by side; HA_LA_TC_SEGMENTS=1|2|4|8 fixes the number of segments a head's
- * chunk sequence is split into.  Production callers leave them unset.
+ * chunk sequence is split into.  Production callers leave them unset; a caller that sets one
+ * does so before it asks for the workspace size (the size follows the plan, and a call whose
+ * plan needs more than it was given returns HA_LA_ERR_WORKSPACE).
  */
 #ifndef HA_LA_H_
 #define HA_LA_H_

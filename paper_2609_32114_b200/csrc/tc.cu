@@ -206,11 +206,12 @@ bool tc_supported(const Problem& p) {
   return p.dtype == HA_LA_BF16 && p.dk == 128 && p.dv == 128;
 }
 
-// (the largest segment count the planner may pick, so that the environment switches cannot outgrow a workspace
-// that was sized before they were set)
+// Images plus, when the planner cuts the sequences into segments, the segment scratch for that many.  (The call
+// checks the caller's size against this same function, so an environment switch that is changed between sizing and
+// calling ends in HA_LA_ERR_WORKSPACE, not in an overrun.)
 size_t tc_workspace_bytes(const Problem& p) {
   const size_t img = tc_ws_bytes_for((size_t)p.max_chunks * p.HV, p.variant == HA_LA_KDA);
-  return img + tc_seg_bytes((size_t)p.N * p.HV, 8, (size_t)p.T_total, p.HV);
+  return img + tc_seg_bytes((size_t)p.N * p.HV, plan_tc(p).nseg, (size_t)p.T_total, p.HV);
 }
 
 int tc_num_launches(const Problem& p) { return plan_tc(p).nseg > 1 ? 4 : 2; }
