@@ -118,3 +118,29 @@ def test_launch_plan_for_the_benchmark_shapes(lib, monkeypatch):
     with pytest.raises(ha.HaLaError):
         plan(_args(dk=96))
     assert lib.ha_la_prefill_launch_plan(ctypes.byref(_args()), None, None) == binding.HA_LA_ERR_INVALID_ARG
+
+
+def test_workspace_follows_the_segment_plan(lib, monkeypatch):
+    """The segment scratch is part of the workspace only when the plan cuts the sequences: b, the transition
+    matrix (fp32) and the start state (bf16) per (sequence, V-head, segment), plus one bf16 row of 128 channels
+    per (token, V-head), rounded up to 1 KiB."""
+    for var in ("HA_LA_TC_NV", "HA_LA_TC_OVERLAP", "HA_LA_FORCE_SIMT", "HA_LA_TC_SEGMENTS"):
+        monkeypatch.delenv(var, raising=False)
+    wb, nseg = ha.ha_la_prefill_workspace_bytes, ha.ha_la_prefill_num_segments
+    a = _args()                                            # the headline shape: one segment
+    assert nseg(a) == 1
+    plain = wb(a)
+    monkeypatch.setenv("HA_LA_TC_SEGMENTS", "4")
+    assert nseg(a) == 4
+    rows = -(-4096 * 16 * 128 * 2 // 1024) * 1024
+    assert wb(a) - plain == 16 * 4 * 128 * 128 * 10 + rows
+    monkeypatch.setenv("HA_LA_TC_SEGMENTS", "1")
+    assert wb(a) == plain
+    monkeypatch.delenv("HA_LA_TC_SEGMENTS")
+    long2 = _args(seqlen=16384, hk=2, hv=2)                # few heads, long row: the planner cuts it itself
+    n = nseg(long2)
+    assert n > 1
+    monkeypatch.setenv("HA_LA_TC_SEGMENTS", "1")
+    one = wb(long2)
+    monkeypatch.delenv("HA_LA_TC_SEGMENTS")
+    assert wb(long2) - one == 2 * n * 128 * 128 * 10 + 16384 * 2 * 128 * 2
