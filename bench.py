@@ -373,7 +373,7 @@ def decode_bench(args, rank, local_rank, world):
 
 def measure(ha, helpers, w, inp, steps, warmup, dev, local_rank, dist, peaks, world, sample_clocks=True):
     """Device-timed steps of ha_la_prefill on workload `w`: `steps` timed calls after max(warmup, 3) untimed ones,
-    one CUDA-event pair per step on the launching stream, every step on a different resident input/output set."""
+    between CUDA events on the launching stream, every step on a different resident input/output set."""
     import torch
 
     T, N = inp["T"], inp["N"]
@@ -419,26 +419,48 @@ def measure(ha, helpers, w, inp, steps, warmup, dev, local_rank, dist, peaks, wo
     barrier()
     check_status("during warm-up")
 
-    # ---- timed region: exactly `steps` steps, device-timed per step (flush, if any, sits outside the events)
+    # ---- timed region: exactly `steps` steps back to back on the launching stream between one pair of CUDA events
+    # (every step works on another resident set, together larger than twice the L2).  Workloads so small that L2 has
+    # to be flushed between steps are timed step by step instead, the flush outside the events.
     sampler = ClockSampler(local_rank) if sample_clocks else None
     if sampler:
         sampler.start()
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    e_all = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
     barrier()
     t_wall = time.perf_counter()
-    for i in range(steps):
-        if flush is not None:
+    if flush is None:
+        e_all[0].record(stream)
+        for i in range(steps):
+            step(i)
+        e_all[1].record(stream)
+    else:
+        for i in range(steps):
             flush.fill_(i & 0xff)
-        evs[i][0].record(stream)
-        step(i)
-        evs[i][1].record(stream)
+            evs[i][0].record(stream)
+            step(i)
+            evs[i][1].record(stream)
     barrier()
     t_wall = time.perf_counter() - t_wall
     check_status("during the timed steps")
     last = sets[(steps - 1) % R][1]
     last_out = {"o": last["o"].clone(), "hT": last["hT"].clone()}     # what the last timed step wrote
-    step_ms = [a.elapsed_time(b) for a, b in evs]
-    total_ms = max_over_ranks(dist, float(np.sum(step_ms)), dev)
+    if flush is None:
+        total_local = e_all[0].elapsed_time(e_all[1])
+        # the spread of single steps: the same steps once more, one event pair each (an event between two calls costs
+        # a couple of microseconds and keeps the next call's set-up from running under this call's tail, so these
+        # are a little longer than the steps of the timed region)
+        for i in range(steps):
+            evs[i][0].record(stream)
+            step(i)
+            evs[i][1].record(stream)
+        barrier()
+        check_status("during the single-step timing")
+        step_ms = [a.elapsed_time(b) for a, b in evs]
+    else:
+        step_ms = [a.elapsed_time(b) for a, b in evs]
+        total_local = float(np.sum(step_ms))
+    total_ms = max_over_ranks(dist, float(total_local), dev)
     ms_per_step = total_ms / steps
     value = job_throughput(world, T, ms_per_step)
 
@@ -668,7 +690,10 @@ def main():
                            "parallelism": "replicas (independent batch per GPU, no collective)" if world > 1 else "1 GPU"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": m["launches_per_step"] * args.steps,
                 "roofline": roofline, "parity": parity, "cpu_baseline": cpu, "other_workloads": others,
-                "wall_s_timed_region": m["wall_s"]}
+                "wall_s_timed_region": m["wall_s"],
+                "timing": ("ms_per_step: the timed steps back to back between one pair of CUDA events on the launching stream; "
+                           "median/min/max: the same steps again with one event pair each" if not m["flushed"] else
+                           "one CUDA-event pair per step, the L2 flush outside the events")}
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

@@ -147,6 +147,14 @@ constexpr int BAR_U_READY = 2;   // the U~ writers (half of them) arrive, MMA wa
 constexpr int BAR_O_FREE = 3;    // output threads: the previous tile store has read the staging tile
 constexpr int BAR_O_FULL = 4;    // output threads: the staging tile is written
                                  // (the whole-head kernel has two tiles: ids 3, 4 for tile 0 and 5, 6 for tile 1)
+// A chain CTA lets the stream's next programmatic dependent be scheduled when it has this many chunks left (CTAs
+// with fewer chunks: when they exit).  That kernel -- the next call's prep kernel, or the segment fix-up -- then
+// gets through its launch and set-up under the tail of this one and waits at its griddepcontrol.wait for this
+// grid to complete; only kernels launched with the programmatic attribute react.
+constexpr int kTailChunks = 6;
+__device__ __forceinline__ void launch_dependents_early() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 __device__ __forceinline__ void named_arrive(int id, int count) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
@@ -331,6 +339,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
       const uint8_t* stage = sm + st * Cfg::kStageB;
       const int L = min(kChunk, len - c * kChunk);
       const uint32_t ph = c & 1;
+      if (c == nchunks - kTailChunks) launch_dependents_early();
 
       HA_PROF(chain, 8 * c + 0);
       mbar_wait(&bar_full[st], (c / S) & 1, abort_flag, p.spin_limit);
@@ -698,6 +707,7 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
       const int st = c % S;
       const uint8_t* stage = sm + st * Cfg::kStageB;
       const uint32_t ph = c & 1;
+      if (c == nchunks - kTailChunks) launch_dependents_early();
       HA_PROF(chain, 8 * c + 0);
       mbar_wait(&bar_full[st], (c / S) & 1, abort_flag, p.spin_limit);
       HA_PROF(chain, 8 * c + 1);

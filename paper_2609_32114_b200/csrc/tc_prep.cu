@@ -283,6 +283,11 @@ tc_prep_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
+  // This kernel is launched as a programmatic dependent of whatever precedes it in the stream; when that is the
+  // previous call's chain kernel, which lets its dependents go a few chunks before its end, everything above ran
+  // under that kernel's tail.  Nothing of this call has been read or written so far: wait for the stream's earlier
+  // work to complete here.  (A no-op after a kernel that triggers nothing early, or without the launch attribute.)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // Every CTA of this grid is running now: a dependent launch (the chain kernel) may be scheduled.  It either
   // waits for this grid to finish or consumes chunks as they are published.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -1062,8 +1067,17 @@ static cudaError_t launch_prep_variant(const PrepParams& pp, const CUtensorMap& 
                                        const CUtensorMap& mv, long long grid, cudaStream_t stream) {
   const int smem = KDA ? kPrepSmemKda : kGroups<KDA> * kGroupSmem;
   timer_mark(stream, "tc_prep");
-  tc_prep_kernel<KDA><<<(unsigned)grid, KDA ? kKdaThreads : kPrepThreads * kGroups<KDA>, smem, stream>>>(mq, mk, mv, pp);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(KDA ? kKdaThreads : kPrepThreads * kGroups<KDA>);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = g_timer ? 0 : 1;                        // (per-kernel timing wants one kernel at a time)
+  return cudaLaunchKernelEx(&cfg, tc_prep_kernel<KDA>, mq, mk, mv, pp);
 }
 
 // Sets the kernel's attributes, which also loads it.  Must run before ANY kernel of a concurrent launch is
