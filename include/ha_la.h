@@ -30,6 +30,13 @@
  *   - ha_la_prefill enqueues kernels on the given CUDA stream and returns
  *     without synchronising.  It allocates no device memory and keeps no
  *     pointer after it returns; the args struct is read during the call only.
+ *   - Stream order holds as for any kernel: the call sees what earlier work on the
+ *     stream wrote, later work sees its outputs.  The tensor-core kernels use
+ *     programmatic dependent launch among themselves and let the stream's next
+ *     kernel be scheduled shortly before they end; that only concerns a following
+ *     kernel launched with the programmatic-serialization attribute, which -- as
+ *     CUDA requires of such kernels -- waits for its grid dependency before it
+ *     touches anything this call reads or writes.
  *   - Every entry point returns an ha_la_status; nothing throws or aborts.
  *   - Problems found on the device (a wait that ran out, an index out of
  *     range) are written as a non-zero code to *status_word, which the caller
