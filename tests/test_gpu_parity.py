@@ -159,6 +159,46 @@ def test_split_resume_and_in_place_state():
     assert helpers.rel_max_err(state.cpu().numpy()[0:1].reshape(h_orc.shape), h_orc) <= 2e-2
 
 
+@pytest.mark.parametrize("overlap", ["0", "2"])
+@pytest.mark.parametrize("variant", ["gdn", "kda"])
+def test_dependent_calls_queued_with_nothing_between_them(variant, overlap, monkeypatch):
+    """A sequence prefilled piece by piece, the state handed on in place (h0 = hT = one buffer), every call
+    prepared beforehand and then queued directly behind the previous one: the next call's first kernel is
+    launched and set up under the previous call's tail and must still see that call's state.  The whole
+    round is repeated so that the first piece follows the last piece of the round before."""
+    import torch
+    import paper_2609_32114_b200 as ha
+
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", overlap)
+    base = W["gdn_layer_4k"] if variant == "gdn" else W["kda_8k"]
+    w = synth.shrink(base, seq_lens=[2560], hk=2, hv=2, gate_shift=-3.0)      # slow decay: the state matters
+    inp = synth.make_inputs(w, seed=131)
+    d = helpers.to_device(inp)
+    pieces = [(0, 640), (640, 1024), (1024, 1100), (1100, 2048), (2048, 2560)]
+    state = torch.zeros((1, 2, 128, 128), dtype=torch.float32, device="cuda")
+    o = torch.zeros_like(d["v"])
+    calls = []
+    for a, b in pieces:
+        cut = lambda t: t[:, a:b].contiguous()
+        o_piece = torch.empty_like(cut(d["v"]))
+        args, keep = ha.prepare_args(cut(d["q"]), cut(d["k"]), cut(d["v"]), cut(d["g"]), cut(d["beta"]),
+                                     variant=variant, h0=state, hT=state, o=o_piece)
+        calls.append((args, keep, a, b))
+    stream = torch.cuda.current_stream().cuda_stream
+    torch.cuda.synchronize()
+    for rnd in range(3):
+        state.zero_()
+        for args, keep, a, b in calls:                       # nothing but these launches goes on the stream
+            assert ha.ha_la_prefill_raw(args, stream) == 0
+    torch.cuda.synchronize()
+    for args, keep, a, b in calls:
+        assert int(keep["status_word"].item()) == 0
+        o[:, a:b] = keep["o"]
+    o_ref, h_ref = helpers.run_oracle(inp)
+    assert helpers.rel_max_err(o[0].float().cpu().numpy(), o_ref) <= 2e-2
+    assert helpers.rel_max_err(state.cpu().numpy().reshape(h_ref.shape), h_ref) <= 2e-2
+
+
 def test_run_to_run_determinism():
     w = synth.shrink(W["gdn_layer_4k"], seq_lens=[777], hk=2, hv=4)
     inp = synth.make_inputs(w, seed=23)
