@@ -9,8 +9,8 @@
 //     h_{s+1} = Phi_s h_s + b_s          (h_1 is segment 0's end state: it started from the real h0)
 //     o_t    += R_t h_s                  for every token t of segment s
 // Two small kernels do that:
-//   seg_fix_kernel   per (sequence, V-head) and tile of 16 state columns: the S - 1 products in turn, fp32 on the
-//                    CUDA cores (128 x 128 x 16 each); writes hT and a bf16 copy of every h_s;
+//   seg_fix_kernel   per (sequence, V-head) and tile of 32 state columns: the S - 1 products in turn, TF32 on the
+//                    legacy tensor path (128 x 128 x 32 each); writes hT and a bf16 copy of every h_s;
 //   seg_out_kernel   per (chunk of a later segment, V-head): o += R h_s on the legacy tensor path (wmma bf16,
 //                    fp32 accumulation), 64 x 128 x 128; chunk-parallel, no dependency between CTAs.
 #include <mma.h>
