@@ -174,7 +174,7 @@ TcPlan plan_tc(const Problem& p) {
   // sequence's chain is cut into nseg segments that run at once; a later segment costs three times the columns of
   // the first (its own from a zero state plus 128 transition columns), so it only pays while all those CTAs have an
   // SM each, i.e. for few heads and long sequences.  Costs measured on B200: the chain's per-chunk times above,
-  // 7 us + 5.5 us per further segment for the start states (S - 1 products of 128^3 in turn) and 9 us + 25 ns per
+  // 7 us + 3.1 us per further segment for the start states (S - 1 products of 128^3 in turn) and 9 us + 15 ns per
   // corrected chunk-head for the outputs.
   int forced_seg = 0;
   if (const char* e = getenv("HA_LA_TC_SEGMENTS")) {
@@ -192,7 +192,7 @@ TcPlan plan_tc(const Problem& p) {
         const double cpseg = (double)(long long)((longest + nseg - 1) / nseg);
         const double waves = (double)((ctas + sms - 1) / sms);
         const double later = items * (1.0 - 1.0 / nseg);
-        const double t = prep_us + waves * cpseg * per_chunk_us[w] + (7.0 + 5.5 * (nseg - 1)) + (9.0 + 0.025 * later);
+        const double t = prep_us + waves * cpseg * per_chunk_us[w] + (7.0 + 3.1 * (nseg - 1)) + (9.0 + 0.015 * later);
         if (t < best || (forced_seg && plan.nseg != forced_seg)) { best = t; plan = TcPlan{widths[w], false, nseg}; }
       }
     }
