@@ -521,6 +521,32 @@ def measure(ha, helpers, w, inp, steps, warmup, dev, local_rank, dist, peaks, wo
                 launches_per_step=ha.ha_la_prefill_num_launches(sets[0][0]), path=ha.ha_la_prefill_path(sets[0][0]))
 
 
+def profile_range(ha, helpers, w, inp, warmup, dev):
+    """One call of ha_la_prefill between cudaProfilerStart and cudaProfilerStop, after `warmup` untimed calls."""
+    import torch
+
+    d = helpers.to_device(inp, dev)
+    a, keep = ha.prepare_args(d["q"], d["k"], d["v"], d["g"], d["beta"], variant=w.variant, h0=d["h0"],
+                              cu_seqlens=d["cu_seqlens"], max_seqlen=d["max_seqlen"])
+    sptr = torch.cuda.current_stream(dev).cuda_stream
+    for _ in range(warmup):
+        ha.ha_la_prefill_raw(a, sptr)
+    flush = torch.empty(3 * L2_BYTES, dtype=torch.uint8, device=dev)
+    flush.fill_(1)                                       # the profiled call starts from a cold L2
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()
+    e0.record()
+    rc = ha.ha_la_prefill_raw(a, sptr)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    torch.cuda.profiler.stop()
+    nv, conc = ha.ha_la_prefill_launch_plan(a)
+    print(json.dumps({"profile_range": w.name, "tokens": inp["T"], "rc": rc, "status": int(keep["status_word"].item()),
+                      "ms": e0.elapsed_time(e1), "slice_width": nv, "side_by_side": bool(conc),
+                      "alg_bytes": synth.algorithmic_bytes(w, inp["T"], inp["N"])}), flush=True)
+
+
 def parity_of(helpers, inp, out):
     """o and hT in `out` (device tensors a step wrote) against the oracle on every (sequence, V-head) pair."""
     w = inp["workload"]
@@ -545,6 +571,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parity", action="store_true", help="skip the oracle comparison of the timed outputs")
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the short timings of the other workloads")
+    ap.add_argument("--seq-len", type=int, default=0,
+                    help="profiling captures: the same workload with sequences of this length (equal-length workloads)")
+    ap.add_argument("--profile-range", action="store_true",
+                    help="profiling captures: warm up, bracket ONE call with cudaProfilerStart/Stop, print its device "
+                         "time and exit (for `ncu --replay-mode range`, which measures the call's kernels together)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -555,6 +586,10 @@ def main():
     if args.workload in DECODE_WORKLOADS:
         return decode_bench(args, rank, local_rank, world)
     w = synth.WORKLOADS[args.workload]
+    if args.seq_len > 0:
+        if w.seq_lens is None:
+            raise SystemExit("--seq-len applies to the equal-length workloads")
+        w = synth.shrink(w, seq_lens=[args.seq_len] * len(w.seq_lens), hk=w.hk, hv=w.hv)
     if args.impl == "reference":
         if rank == 0:
             run_reference(args, synth.make_inputs(w), rank)
@@ -577,6 +612,8 @@ def main():
     # every rank draws its own batch of the same workload (weak scaling over independent batches)
     inp = synth.make_inputs(w, seed=rank_seed(rank))
     T, N = inp["T"], inp["N"]
+    if args.profile_range:
+        return profile_range(ha, helpers, w, inp, max(args.warmup, 3), dev)
     peaks = load_peaks()
     m = measure(ha, helpers, w, inp, args.steps, args.warmup, dev, local_rank, dist, peaks, world)
     sets, R, base, stream, sptr = m["sets"], m["R"], m["base"], m["stream"], m["sptr"]

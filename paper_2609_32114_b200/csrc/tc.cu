@@ -91,14 +91,15 @@ constexpr int kMaxDevices = 64;
 constexpr uint32_t kDefaultSpinLimit = 4u << 20;      // polls before a device-side bounded wait gives up
 std::atomic<uint32_t> g_calls{0};
 
-// Epoch of a concurrent-mode call: (random per-process tag, never 0) << 32 | call counter.
+// Epoch of a concurrent-mode call: (random per-process tag, never 0) << 40 | call counter << 8; the low byte is zero
+// (the chain kernel's slices count in it).
 int64_t next_epoch() {
   static const uint32_t tag = [] {
     std::random_device rd;
     uint32_t t = rd();
-    return t ? t : 0x9e3779b9u;
+    return (t & 0x7fffffu) ? t : 0x9e3779b9u;
   }();
-  return (int64_t)(((uint64_t)tag << 32) | g_calls.fetch_add(1));
+  return (int64_t)(((uint64_t)(tag & 0x7fffffu) << 40) | ((uint64_t)(uint32_t)g_calls.fetch_add(1) << 8));
 }
 
 // Slice width (value channels per chain CTA) and launch mode, from a cost model measured on B200.

@@ -38,7 +38,8 @@ HA_PROF_DECL(chain)
 
 namespace {
 
-constexpr int chain_threads(int cg) { return (4 * cg + 2) * 32; }   // compute warps + producer warp + MMA warp
+// compute warps + producer warp + MMA warp (+ a clean-up warp in the instances that drop consumed images from L2)
+constexpr int chain_threads(int cg, bool drop) { return (4 * cg + 2 + (drop ? 1 : 0)) * 32; }
 
 template <int NV, int S_> struct ChainCfg {
   static constexpr int kStages = S_;
@@ -56,7 +57,7 @@ template <int NV, int S_> struct ChainCfg {
   static constexpr uint32_t OFF_OUT = OFF_UT + 64 * kRowB;       // bf16 output tile [64][NV], staged for the tile store
   static constexpr uint32_t kSmem = OFF_OUT + 64 * kRowB;
   static constexpr uint32_t OFF_BAR = OFF_SC + 768;              // barriers live in the unused tail of stage 0
-  static_assert(kStageB - OFF_BAR >= (2 * S_ + 2) * 8 + 16, "room for the barriers");
+  static_assert(kStageB - OFF_BAR >= (2 * S_ + 2) * 8 + 16, "room for the barriers and three words");
   static constexpr uint32_t kTmemCols = 2 * NV < 32 ? 32 : 2 * NV;
 };
 
@@ -75,6 +76,7 @@ struct ChainParams {
   int64_t epoch;               // != 0: the prep kernel runs concurrently; wait for ws.flags[cj] == epoch per chunk
                                // == 0: wait for the whole prep grid before the first workspace read
   uint32_t spin_limit;         // polls before a bounded wait gives up (kSpinLimit; a few thousand in the time-out test)
+  int drop_consumed;           // concurrent mode, images larger than half of L2: drop consumed images from L2 (clean-up warp)
   // Segment-parallel state passing (sliced kernels, equal-length rows): a sequence's chunks are cut into `nseg`
   // segments that run at the same time.  Segment 0 starts from h0.  A later segment s runs twice over: its value
   // columns from a ZERO state (provisional outputs into o, end state b_s into seg_b) and 128 "transition" columns
@@ -162,14 +164,14 @@ __device__ __forceinline__ void named_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
-template <int NV, bool KDA, int S, int CG>
-__global__ void __launch_bounds__(chain_threads(CG), 1)
+template <int NV, bool KDA, int S, int CG, bool DROP>
+__global__ void __launch_bounds__(chain_threads(CG, DROP), 1)
 tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_o, ChainParams p) {
   using Cfg = ChainCfg<NV, S>;
   constexpr int NSL = 128 / NV;
   constexpr int NVT = NV / CG;                           // value channels per compute thread
   constexpr int NCOMP = 128 * CG;                        // compute threads
-  constexpr int W_PROD = 4 * CG, W_MMA = 4 * CG + 1;
+  constexpr int W_PROD = 4 * CG, W_MMA = 4 * CG + 1, W_CLEAN = 4 * CG + 2;
   static_assert(NVT % 32 == 0, "column groups are multiples of 32 channels");
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* sm = smem_raw;                                // no static shared memory in this kernel: 1024-aligned
@@ -179,6 +181,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
   uint64_t* bar_mma2 = bar_mma1 + 1;                                        // MMA2 complete
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mma2 + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* consumed = reinterpret_cast<volatile int*>(tmem_slot + 2);   // chunks this CTA is done with
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -209,6 +212,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
     mbar_init(bar_mma1, 1);
     mbar_init(bar_mma2, 1);
     *abort_flag = 0;
+    if constexpr (DROP) *consumed = 0;
     mbar_fence_init();
     prefetch_tmap(&map_k);
     prefetch_tmap(&map_o);
@@ -240,7 +244,7 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
           const int cc = c + lane;
           bool ok = false;
           if (cc < nchunks)
-            ok = *reinterpret_cast<const volatile int64_t*>(p.ws.flags + (size_t)(chunk0 + cc) * p.HV + j) == p.epoch;
+            ok = (*reinterpret_cast<const volatile int64_t*>(p.ws.flags + (size_t)(chunk0 + cc) * p.HV + j) & ~kFlagCountMask) == p.epoch;
           const unsigned m = __ballot_sync(0xffffffffu, ok);
           got = __ffs(~m) - 1;                           // leading published chunks (32 when all are)
           if (got < 0) got = 32;
@@ -301,6 +305,44 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
         for (int ks = 0; ks < 4; ++ks)                    // K = tokens: 16 token rows per step
           umma_ss(TM2, dK + ks * (2048u >> 4), dU + ks * brow_step16<NV>(), id, ks > 0);
         umma_commit(bar_mma2);
+      }
+    }
+  } else if (DROP && warp == W_CLEAN) {
+    // ------------------------------------------------------------ clean-up (concurrent mode, images larger than L2)
+    // The images were written microseconds ago and mostly still sit in L2 as dirty lines.  Once this CTA is done
+    // with a chunk, the U and O_loc rows of its slice -- read by this CTA alone -- are dead, and so are the W / Q~
+    // image (and KDA's K e^{G_L-G} image) when the last slice of the head is done with them: the low byte of the
+    // chunk's flag counts the slices.  Dropping the lines from L2 spares their write-back to HBM.  (Back to back
+    // the lines have long been written back, and a workspace that stays in L2 from call to call is never written
+    // back at all: nothing to gain in either case.)  Nothing waits for this warp; if its wait runs out it stops.
+    if (!trans) {
+      const int lane = tid & 31;
+      for (int c = 0; c < nchunks; ++c) {
+        bool done = false;
+        for (uint32_t it = 0; it < p.spin_limit && !*abort_flag; ++it) {
+          if (*consumed > c) { done = true; break; }
+          __nanosleep(200);
+        }
+        if (!done) break;
+        const size_t cj = (size_t)(chunk0 + c) * p.HV + j;
+        int last = 0;
+        if (lane == 0)
+          last = (atomicAdd(reinterpret_cast<unsigned long long*>(p.ws.flags + cj), 1ull) & kFlagCountMask) == NSL - 1;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        const uint8_t* u0 = p.ws.u + cj * kImgBytes + (size_t)slice * Cfg::kSliceB;
+        const uint8_t* o0 = p.ws.ol + cj * kImgBytes + (size_t)slice * Cfg::kSliceB;
+        for (uint32_t off = lane * 128u; off < Cfg::kSliceB; off += 4096u) {
+          discard_l2_line(u0 + off);
+          discard_l2_line(o0 + off);
+        }
+        if (last) {
+          const uint8_t* w0 = p.ws.wq + cj * 2 * kImgBytes;
+          for (uint32_t off = lane * 128u; off < 2 * kImgBytes; off += 4096u) discard_l2_line(w0 + off);
+          if constexpr (KDA) {
+            const uint8_t* k0 = p.ws.kd + cj * kImgBytes;
+            for (uint32_t off = lane * 128u; off < kImgBytes; off += 4096u) discard_l2_line(k0 + off);
+          }
+        }
       }
     }
   } else {
@@ -420,6 +462,9 @@ tc_chain_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant
       HA_PROF(chain, 8 * c + 4);
       tc_fence_after_sync();
       mbar_arrive(&bar_empty[st]);                       // this thread and both MMAs are done with the stage
+      if constexpr (DROP) {
+        if (tid == 0) *consumed = c + 1;
+      }
 #pragma unroll
       for (int c0 = 0; c0 < NVT; c0 += 32) {
         float d[32];
@@ -554,7 +599,7 @@ tc_chain_t_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
           const int cc = c + lane;
           bool ok = false;
           if (cc < nchunks)
-            ok = *reinterpret_cast<const volatile int64_t*>(p.ws.flags + (size_t)(chunk0 + cc) * p.HV + j) == p.epoch;
+            ok = (*reinterpret_cast<const volatile int64_t*>(p.ws.flags + (size_t)(chunk0 + cc) * p.HV + j) & ~kFlagCountMask) == p.epoch;
           const unsigned m = __ballot_sync(0xffffffffu, ok);
           got = __ffs(~m) - 1;
           if (got < 0) got = 32;
@@ -804,10 +849,10 @@ cudaError_t run_t(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMa
   return cudaLaunchKernelEx(&cfg, kern, *mk, *mo, *cp);
 }
 
-template <int NV, bool KDA, int S, int CG>
-cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMap* mo, int grid, bool dependent,
-                   cudaStream_t stream) {
-  auto kern = tc_chain_kernel<NV, KDA, S, CG>;
+template <int NV, bool KDA, int S, int CG, bool DROP>
+cudaError_t run_nv_inst(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMap* mo, int grid, bool dependent,
+                        cudaStream_t stream) {
+  auto kern = tc_chain_kernel<NV, KDA, S, CG, DROP>;
   constexpr int smem = ChainCfg<NV, S>::kSmem;
   static_assert(smem <= 227 * 1024, "shared memory budget");
   if (!cp) {                                             // configure only (this also loads the kernel)
@@ -820,7 +865,7 @@ cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, const CUtensorM
   // as every prep CTA is running, instead of after the prep grid has drained.
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(chain_threads(CG));
+  cfg.blockDim = dim3(chain_threads(CG, DROP));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -829,6 +874,19 @@ cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, const CUtensorM
   cfg.attrs = attr;
   cfg.numAttrs = dependent ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kern, *mk, *mo, *cp);
+}
+
+// Two instances per width: with and without the clean-up warp (ChainParams::drop_consumed); both are configured.
+template <int NV, bool KDA, int S, int CG>
+cudaError_t run_nv(const ChainParams* cp, const CUtensorMap* mk, const CUtensorMap* mo, int grid, bool dependent,
+                   cudaStream_t stream) {
+  if (!cp) {
+    cudaError_t e = run_nv_inst<NV, KDA, S, CG, false>(cp, mk, mo, grid, dependent, stream);
+    if (e != cudaSuccess) return e;
+    return run_nv_inst<NV, KDA, S, CG, true>(cp, mk, mo, grid, dependent, stream);
+  }
+  return cp->drop_consumed ? run_nv_inst<NV, KDA, S, CG, true>(cp, mk, mo, grid, dependent, stream)
+                           : run_nv_inst<NV, KDA, S, CG, false>(cp, mk, mo, grid, dependent, stream);
 }
 
 // Slices of 64 value channels are worked on by two column groups of compute warps.
@@ -855,6 +913,12 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
   cp.ws = ws; cp.HK = p.HK; cp.HV = p.HV; cp.scale = p.scale; cp.status = a.status_word;
   cp.epoch = epoch;
   cp.spin_limit = spin_limit;
+  {
+    int dev = 0, l2 = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev);
+    const size_t images = (size_t)p.max_chunks * p.HV * 4 * kImgBytes;
+    cp.drop_consumed = epoch != 0 && sg.nseg == 1 && images > (size_t)l2 / 2;
+  }
   cp.nseg = sg.nseg; cp.seg_b = sg.seg_b; cp.seg_phi = sg.seg_phi; cp.r_out = sg.r;
   const int grid = p.N * p.HV * (128 / nv) * (2 * sg.nseg - 1);
   if (grid == 0) return cudaSuccess;

@@ -23,6 +23,10 @@ namespace ha_la {
 constexpr size_t kImgBytes = 128 * 64 * 2;     // 16 KiB
 constexpr int kScFloats = 192;
 
+// A chunk's ready flag holds the call's epoch (low byte zero) when the prep kernel has published it; the chain
+// kernel's slices then count themselves off in the low byte as they finish with the chunk.
+constexpr long long kFlagCountMask = 0xff;
+
 struct TcWorkspace {
   uint8_t* wq;
   uint8_t* u;

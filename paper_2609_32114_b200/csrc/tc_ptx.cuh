@@ -119,6 +119,11 @@ __device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes
   asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(src)), "r"(bytes) : "memory");
 }
 
+// Drops one 128-byte line from L2 without writing it back; its contents become undefined (scratch only).
+__device__ __forceinline__ void discard_l2_line(const void* p) {
+  asm volatile("discard.global.L2 [%0], 128;" ::"l"(reinterpret_cast<uint64_t>(p)) : "memory");
+}
+
 // 1-D bulk copy shared -> global (same alignment rules).  One thread issues, commits the group and,
 // before the shared buffer is reused or the CTA exits, waits until the group has been read.
 __device__ __forceinline__ void bulk_store(void* gdst, const void* ssrc, uint32_t bytes) {

@@ -302,6 +302,36 @@ def test_full_size_all_heads(name):
     print(name, res)
 
 
+@pytest.mark.parametrize("variant,nv,hv", [("gdn", 32, 16), ("gdn", 64, 16), ("kda", 64, 32), ("kda", 32, 16)])
+def test_consumed_images_dropped_from_l2(variant, nv, hv, monkeypatch):
+    """Side by side with operand images larger than half of L2, the chain kernel drops the images it has consumed
+    from L2 (a slice its own rows, the last slice of a head the shared ones, counted in the chunk's flag): every
+    head against the oracle, with four slices (32 channels) and two (64) per head, both variants; twice in a row
+    on one workspace, so that the second call finds the first call's counts in the flags."""
+    import torch
+    import paper_2609_32114_b200 as ha
+
+    monkeypatch.setenv("HA_LA_TC_NV", str(nv))
+    monkeypatch.setenv("HA_LA_TC_OVERLAP", "2")
+    monkeypatch.setenv("HA_LA_TC_SEGMENTS", "1")
+    base = W["gdn_layer_4k"] if variant == "gdn" else W["kda_8k"]
+    w = synth.shrink(base, seq_lens=[8192], hk=hv, hv=hv, h0_std=0.02)      # 128 chunks x hv heads x 64.8 KiB
+    inp = synth.make_inputs(w, seed=151 + nv)
+    d = helpers.to_device(inp)
+    a, keep = ha.prepare_args(d["q"], d["k"], d["v"], d["g"], d["beta"], variant=variant, h0=d["h0"])
+    assert ha.ha_la_prefill_launch_plan(a) == (nv, True)
+    stream = torch.cuda.current_stream().cuda_stream
+    o_ref, h_ref = helpers.run_oracle(inp)
+    for rep in range(2):
+        keep["o"].zero_()
+        keep["hT"].zero_()
+        assert ha.ha_la_prefill_raw(a, stream) == 0
+        torch.cuda.synchronize()
+        assert int(keep["status_word"].item()) == 0
+        assert helpers.rel_max_err(keep["o"][0].float().cpu().numpy(), o_ref) <= 2e-2
+        assert helpers.rel_max_err(keep["hT"].cpu().numpy().reshape(h_ref.shape), h_ref) <= 2e-2
+
+
 @pytest.mark.parametrize("variant", ["gdn", "kda"])
 @pytest.mark.parametrize("nv", [32, 64, 128])
 def test_tc_every_slice_width(nv, variant, monkeypatch):
