@@ -76,7 +76,7 @@ struct ChainParams {
   int64_t epoch;               // != 0: the prep kernel runs concurrently; wait for ws.flags[cj] == epoch per chunk
                                // == 0: wait for the whole prep grid before the first workspace read
   uint32_t spin_limit;         // polls before a bounded wait gives up (kSpinLimit; a few thousand in the time-out test)
-  int drop_consumed;           // concurrent mode, images larger than half of L2: drop consumed images from L2 (clean-up warp)
+  int drop_consumed;           // concurrent mode, images larger than L2: drop consumed images from L2 (clean-up warp)
   // Segment-parallel state passing (sliced kernels, equal-length rows): a sequence's chunks are cut into `nseg`
   // segments that run at the same time.  Segment 0 starts from h0.  A later segment s runs twice over: its value
   // columns from a ZERO state (provisional outputs into o, end state b_s into seg_b) and 128 "transition" columns
@@ -917,7 +917,7 @@ cudaError_t launch_tc_chain(const Problem& p, const ha_la_prefill_args& a, PlanV
     int dev = 0, l2 = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev);
     const size_t images = (size_t)p.max_chunks * p.HV * 4 * kImgBytes;
-    cp.drop_consumed = epoch != 0 && sg.nseg == 1 && images > (size_t)l2 / 2;
+    cp.drop_consumed = epoch != 0 && sg.nseg == 1 && images > (size_t)l2;
   }
   cp.nseg = sg.nseg; cp.seg_b = sg.seg_b; cp.seg_phi = sg.seg_phi; cp.r_out = sg.r;
   const int grid = p.N * p.HV * (128 / nv) * (2 * sg.nseg - 1);

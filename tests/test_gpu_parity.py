@@ -304,7 +304,7 @@ def test_full_size_all_heads(name):
 
 @pytest.mark.parametrize("variant,nv,hv", [("gdn", 32, 16), ("gdn", 64, 16), ("kda", 64, 32), ("kda", 32, 16)])
 def test_consumed_images_dropped_from_l2(variant, nv, hv, monkeypatch):
-    """Side by side with operand images larger than half of L2, the chain kernel drops the images it has consumed
+    """Side by side with operand images larger than L2, the chain kernel drops the images it has consumed
     from L2 (a slice its own rows, the last slice of a head the shared ones, counted in the chunk's flag): every
     head against the oracle, with four slices (32 channels) and two (64) per head, both variants; twice in a row
     on one workspace, so that the second call finds the first call's counts in the flags."""
