@@ -37,6 +37,10 @@
  *     kernel launched with the programmatic-serialization attribute, which -- as
  *     CUDA requires of such kernels -- waits for its grid dependency before it
  *     touches anything this call reads or writes.
+ *   - ha_la_prefill and ha_la_decode may be captured into a CUDA graph by stream
+ *     capture and replayed on new contents of the same buffers; pointers, sizes
+ *     and the launch plan are frozen at capture.  (ha_la_prefill_timed blocks and
+ *     cannot be captured.)
  *   - Every entry point returns an ha_la_status; nothing throws or aborts.
  *   - Problems found on the device (a wait that ran out, an index out of
  *     range) are written as a non-zero code to *status_word, which the caller

@@ -257,6 +257,20 @@ cudaError_t launch_tc(const Problem& p, const ha_la_prefill_args& a, PlanView pl
     epoch = next_epoch();
     reserved_sms = p.N * p.HV * (128 / nv);              // a chain CTA fills its SM
   }
+  if (concurrent) {
+    // A call captured into a CUDA graph is replayed with the epoch it was captured with, and the flags its last
+    // replay left behind carry exactly that epoch: the chain kernel would run ahead of the prep kernel on stale
+    // images.  Under capture the flags are therefore cleared first (a memset node, replayed with the rest).
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess) {
+      (void)cudaGetLastError();
+      cs = cudaStreamCaptureStatusNone;
+    }
+    if (cs == cudaStreamCaptureStatusActive) {
+      const cudaError_t me = cudaMemsetAsync(ws.flags, 0, ncj * sizeof(int64_t), stream);
+      if (me != cudaSuccess) return me;
+    }
+  }
   cudaError_t e = launch_tc_prep(p, a, plan, ws, mq, mk, mv, epoch, reserved_sms, stream);
   if (e != cudaSuccess) return e;
   e = launch_tc_chain(p, a, plan, ws, mk, mo, nv, epoch, /*dependent=*/g_timer == nullptr, kDefaultSpinLimit, sg, stream);

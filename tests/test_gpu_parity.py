@@ -199,6 +199,50 @@ def test_dependent_calls_queued_with_nothing_between_them(variant, overlap, monk
     assert helpers.rel_max_err(state.cpu().numpy().reshape(h_ref.shape), h_ref) <= 2e-2
 
 
+@pytest.mark.parametrize("shape", ["side_by_side", "back_to_back", "segments", "packed"])
+def test_call_captured_in_a_cuda_graph(shape):
+    """A call captured by stream capture and replayed on new contents of the same buffers: every replay must equal
+    an ordinary call on those contents.  (Side by side, the ready flags a replay leaves behind carry the very
+    epoch the next replay runs with: under capture the call clears them first.)"""
+    import torch
+    import paper_2609_32114_b200 as ha
+
+    kw = {"side_by_side": dict(seq_lens=[2048], hk=16, hv=16), "back_to_back": dict(seq_lens=[1000], hk=4, hv=4),
+          "segments": dict(seq_lens=[8192], hk=2, hv=2), "packed": dict(seq_lens=[300, 0, 700, 64], hk=2, hv=4, varlen=True)}[shape]
+    w = synth.shrink(W["gdn_varlen"] if shape == "packed" else W["gdn_layer_4k"], h0_std=0.02, **kw)
+    dev = [helpers.to_device(synth.make_inputs(w, seed=s)) for s in (171, 172)]
+    buf = {k: (v.clone() if hasattr(v, "clone") else v) for k, v in dev[0].items()}
+    a, keep = ha.prepare_args(buf["q"], buf["k"], buf["v"], buf["g"], buf["beta"], variant=w.variant, h0=buf["h0"],
+                              cu_seqlens=buf["cu_seqlens"], max_seqlen=buf["max_seqlen"])
+    nv, conc = ha.ha_la_prefill_launch_plan(a)
+    assert conc == (shape == "side_by_side") and (ha.ha_la_prefill_num_segments(a) > 1) == (shape == "segments")
+    names = [k for k in ("q", "k", "v", "g", "beta", "h0") if buf[k] is not None]
+    side = torch.cuda.Stream()
+    ref = []
+    with torch.cuda.stream(side):
+        for d in dev:                                        # ordinary calls: the references (and the warm-up)
+            for k in names:
+                buf[k].copy_(d[k])
+            assert ha.ha_la_prefill_raw(a, side.cuda_stream) == 0
+            side.synchronize()
+            ref.append((keep["o"].clone(), keep["hT"].clone()))
+    assert not torch.equal(ref[0][0], ref[1][0])
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        assert ha.ha_la_prefill_raw(a, torch.cuda.current_stream().cuda_stream) == 0
+    for rep in range(6):
+        which = (rep + 1) % 2
+        for k in names:
+            buf[k].copy_(dev[which][k])
+        keep["o"].zero_()
+        keep["hT"].zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert int(keep["status_word"].item()) == 0
+        assert torch.equal(keep["o"], ref[which][0]) and torch.equal(keep["hT"], ref[which][1]), f"replay {rep}"
+    helpers.check_parity(synth.make_inputs(w, seed=171))     # ... and the ordinary call equals the oracle
+
+
 def test_run_to_run_determinism():
     w = synth.shrink(W["gdn_layer_4k"], seq_lens=[777], hk=2, hv=4)
     inp = synth.make_inputs(w, seed=23)
