@@ -376,6 +376,18 @@ def test_consumed_images_dropped_from_l2(variant, nv, hv, monkeypatch):
         assert helpers.rel_max_err(keep["hT"].cpu().numpy().reshape(h_ref.shape), h_ref) <= 2e-2
 
 
+def test_tensors_beyond_two_gib():
+    """One 270,000-token sequence with 32 V-heads on one q/k head: v and o are 2.2 GB each, so element offsets pass
+    2^30 and byte offsets 2^31 (index arithmetic in 32 bits would wrap), the workspace is 8.8 GB, and a ragged last
+    chunk sits at the far end.  Every head against the oracle (about a minute, half of it drawing the inputs).
+    Run once by hand at 530,000 tokens (4.3 GB per tensor, past 2^31 elements) and for KDA with a 4.4 GB gate
+    tensor: both within the same tolerance."""
+    w = synth.shrink(W["gdn_gva_16k"], seq_lens=[270000], hk=1, hv=32, h0_std=0.02)
+    inp = synth.make_inputs(w, seed=5)
+    assert inp["v"].size * 2 > 2 ** 31
+    helpers.check_parity(inp)
+
+
 @pytest.mark.parametrize("variant", ["gdn", "kda"])
 @pytest.mark.parametrize("nv", [32, 64, 128])
 def test_tc_every_slice_width(nv, variant, monkeypatch):
