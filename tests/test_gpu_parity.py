@@ -243,6 +243,44 @@ def test_call_captured_in_a_cuda_graph(shape):
     helpers.check_parity(synth.make_inputs(w, seed=171))     # ... and the ordinary call equals the oracle
 
 
+@pytest.mark.parametrize("seed", [21, 22, 23])
+def test_random_shapes_and_launch_modes(seed, monkeypatch):
+    """A seeded sweep over what the planner can be made to do: variant, packed or batched sequences with lengths
+    around the chunk boundaries (empty ones included), head counts and grouping, gate strength, initial state,
+    slice width, launch mode, segment count, output scale -- each case against the oracle."""
+    import random
+
+    rng = random.Random(seed)
+    for it in range(14):
+        variant = rng.choice(["gdn", "kda"])
+        nseq = rng.choice([1, 1, 2, 3, 5])
+        lens = [rng.choice([0, 1, 63, 64, 65, 127, 128, 129, 200, 511, 700, 1000, 1537]) for _ in range(nseq)]
+        if sum(lens) == 0:
+            lens[0] = 77
+        hk = rng.choice([1, 2, 4])
+        hv = hk * rng.choice([1, 1, 2])
+        packed = rng.choice([True, True, False])
+        if not packed:
+            lens = [max(lens[0], 1)] * nseq
+        base = W["gdn_varlen"] if variant == "gdn" else W["kda_8k"]
+        w = synth.shrink(base, seq_lens=lens, hk=hk, hv=hv, gate_shift=rng.choice([-4.0, -2.0, 0.0, 2.0]),
+                         h0_std=rng.choice([0.0, 0.02]), varlen=packed)
+        nv = rng.choice(["", "32", "64", "128"])
+        ov = rng.choice(["", "0", "2"])
+        sg = rng.choice(["", "", "2", "4", "8"]) if nv != "128" else ""
+        for key, val in (("HA_LA_TC_NV", nv), ("HA_LA_TC_OVERLAP", ov), ("HA_LA_TC_SEGMENTS", sg)):
+            if val:
+                monkeypatch.setenv(key, val)
+            else:
+                monkeypatch.delenv(key, raising=False)
+        inp = synth.make_inputs(w, seed=1000 * seed + it)
+        try:
+            helpers.check_parity(inp, scale=rng.choice([1.0, 0.5]))
+        except AssertionError as e:
+            raise AssertionError(f"case {it}: {variant} lens={lens} hk={hk} hv={hv} packed={packed} nv={nv!r} "
+                                 f"overlap={ov!r} segments={sg!r}: {e}") from e
+
+
 def test_run_to_run_determinism():
     w = synth.shrink(W["gdn_layer_4k"], seq_lens=[777], hk=2, hv=4)
     inp = synth.make_inputs(w, seed=23)
